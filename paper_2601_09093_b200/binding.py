@@ -1,0 +1,230 @@
+"""ctypes binding of libstep.so - argument marshalling only.
+
+Function names mirror the C header (include/step.h).  PyTorch is used for device memory and
+streams; every step of the hot path runs in the library's CUDA kernels.  There is no CPU
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstep.so")
+
+STEP_OK = 0
+STATUS_NAMES = {0: "STEP_OK", 1: "STEP_ERR_INVALID_ARG", 2: "STEP_ERR_NO_BLOCKS", 3: "STEP_ERR_BAD_TRACE",
+                4: "STEP_ERR_CAPACITY", 5: "STEP_ERR_CUDA", 6: "STEP_ERR_TIMEOUT", 7: "STEP_ERR_BAD_BLOCK"}
+STEP_BF16, STEP_FP32 = 0, 1
+_TORCH_DTYPE = {STEP_BF16: torch.bfloat16, STEP_FP32: torch.float32}
+
+
+class StepError(RuntimeError):
+    def __init__(self, fn, code):
+        super().__init__(f"{fn} failed: {STATUS_NAMES.get(code, code)}")
+        self.code = code
+
+
+class kv_pool_config(C.Structure):
+    _fields_ = [("num_layers", C.c_int), ("num_q_heads", C.c_int), ("num_kv_heads", C.c_int),
+                ("head_dim", C.c_int), ("page_size", C.c_int), ("num_blocks", C.c_int),
+                ("max_traces", C.c_int), ("max_pages_per_trace", C.c_int), ("dtype", C.c_int),
+                ("max_score_rows", C.c_int), ("unscored_score", C.c_float),
+                ("kv_storage", C.c_void_p), ("kv_bytes", C.c_size_t),
+                ("meta_storage", C.c_void_p), ("meta_bytes", C.c_size_t)]
+
+
+class scorer_weights(C.Structure):
+    _fields_ = [("W1", C.c_void_p), ("b1", C.c_void_p), ("w2", C.c_void_p), ("b2", C.c_float),
+                ("D", C.c_int), ("m", C.c_int), ("dtype", C.c_int)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libstep.so (built by paper_2601_09093_b200.build); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2601_09093_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, ip, i = C.c_void_p, C.POINTER(C.c_int), C.c_int
+    L.step_version.restype = C.c_char_p
+    L.kv_pool_required_bytes.argtypes = [C.POINTER(kv_pool_config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.kv_pool_create.argtypes = [C.POINTER(kv_pool_config), C.POINTER(vp)]
+    L.kv_pool_destroy.argtypes = [vp]
+    L.kv_pool_reset.argtypes = [vp, vp]
+    L.kv_pool_fork_prefix.argtypes = [vp, i, i, vp, vp, ip, vp]
+    L.append_kv.argtypes = [vp, vp, i, i, vp, vp, vp]
+    L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
+    L.prune_if_saturated.argtypes = [vp, vp, C.c_float, C.c_float, vp, vp, vp]
+    L.kv_pool_release_traces.argtypes = [vp, vp, i, vp]
+    L.kv_pool_stats.argtypes = [vp, ip, ip, ip, ip, vp]
+    L.kv_pool_device_views.argtypes = [vp] + [C.POINTER(vp)] * 7
+    L.kv_pool_score_views.argtypes = [vp] + [C.POINTER(vp)] * 2
+    L.kv_pool_last_error.argtypes = [vp, C.POINTER(C.c_uint), vp]
+    L.kv_pool_read_kv.argtypes = [vp, i, i, vp, i, vp, vp, vp]
+    L.kv_pool_set_attention_config.argtypes = [vp, i, i]
+    _lib = L
+    return L
+
+
+def _check(fn, code):
+    if code != STEP_OK:
+        raise StepError(fn, code)
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def kv_pool_required_bytes(**geometry):
+    cfg = kv_pool_config(**geometry)
+    kb, mb = C.c_size_t(), C.c_size_t()
+    _check("kv_pool_required_bytes", lib().kv_pool_required_bytes(C.byref(cfg), C.byref(kb), C.byref(mb)))
+    return kb.value, mb.value
+
+
+class KVPool:
+    """Owns the torch tensors behind one step_pool and forwards the C calls."""
+
+    def __init__(self, num_layers, num_q_heads, num_kv_heads, head_dim, page_size, num_blocks, max_traces,
+                 max_pages_per_trace, dtype=STEP_BF16, max_score_rows=0, unscored_score=1.0, device="cuda:0"):
+        self.geometry = dict(num_layers=num_layers, num_q_heads=num_q_heads, num_kv_heads=num_kv_heads,
+                             head_dim=head_dim, page_size=page_size, num_blocks=num_blocks, max_traces=max_traces,
+                             max_pages_per_trace=max_pages_per_trace, dtype=dtype, max_score_rows=max_score_rows,
+                             unscored_score=unscored_score)
+        self.dtype, self.torch_dtype = dtype, _TORCH_DTYPE[dtype]
+        self.device = torch.device(device)
+        kb, mb = kv_pool_required_bytes(**self.geometry)
+        self.kv_bytes, self.meta_bytes = kb, mb
+        with torch.cuda.device(self.device):
+            self.kv_storage = torch.empty(kb, dtype=torch.uint8, device=self.device)
+            self.meta_storage = torch.empty(mb, dtype=torch.uint8, device=self.device)
+            cfg = kv_pool_config(kv_storage=self.kv_storage.data_ptr(), kv_bytes=kb,
+                                 meta_storage=self.meta_storage.data_ptr(), meta_bytes=mb, **self.geometry)
+            h = C.c_void_p()
+            _check("kv_pool_create", lib().kv_pool_create(C.byref(cfg), C.byref(h)))
+        self.handle = h
+        for k, v in self.geometry.items():
+            setattr(self, k, v)
+        self._views = None
+        self.pruned_ids = torch.empty(max_traces, dtype=torch.int32, device=self.device)
+        self.n_pruned = torch.zeros(1, dtype=torch.int32, device=self.device)
+
+    def close(self):
+        if self.handle is not None:
+            lib().kv_pool_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- views into meta_storage as torch tensors (no copies)
+    def _view(self, ptr, count, dtype):
+        off = ptr - self.meta_storage.data_ptr()
+        nbytes = count * torch.empty(0, dtype=dtype).element_size()
+        return self.meta_storage[off:off + nbytes].view(dtype)
+
+    def views(self):
+        if self._views is None:
+            p = [C.c_void_p() for _ in range(7)]
+            _check("kv_pool_device_views", lib().kv_pool_device_views(self.handle, *[C.byref(x) for x in p]))
+            q = [C.c_void_p() for _ in range(2)]
+            _check("kv_pool_score_views", lib().kv_pool_score_views(self.handle, *[C.byref(x) for x in q]))
+            T, NB, MP = self.max_traces, self.num_blocks, self.max_pages_per_trace
+            self._views = dict(
+                block_table=self._view(p[0].value, T * MP, torch.int32).view(T, MP),
+                seq_lens=self._view(p[1].value, T, torch.int32),
+                trace_scores=self._view(p[2].value, T, torch.float32),
+                free_list=self._view(p[3].value, NB, torch.int32),
+                free_count=self._view(p[4].value, 1, torch.int32),
+                refcount=self._view(p[5].value, NB, torch.int32),
+                live=self._view(p[6].value, T, torch.uint8),
+                score_sum=self._view(q[0].value, T, torch.float32),
+                score_cnt=self._view(q[1].value, T, torch.int32))
+        return self._views
+
+    # ---- the calls
+    def reset(self, stream=None):
+        _check("kv_pool_reset", lib().kv_pool_reset(self.handle, _stream(stream)))
+
+    def fork_prefix(self, n_traces, prefix_len, k_prefix, v_prefix, stream=None):
+        ids = (C.c_int * n_traces)()
+        _check("kv_pool_fork_prefix", lib().kv_pool_fork_prefix(self.handle, n_traces, prefix_len, _ptr(k_prefix),
+                                                                _ptr(v_prefix), ids, _stream(stream)))
+        return list(ids)
+
+    def append_kv(self, trace_ids, n_tokens, k_new, v_new, stream=None):
+        _check("append_kv", lib().append_kv(self.handle, _ptr(trace_ids), trace_ids.numel(), n_tokens, _ptr(k_new),
+                                            _ptr(v_new), _stream(stream)))
+
+    def decode_attention(self, layer, q, block_table, seq_lens, out=None, stream=None):
+        n = q.shape[0]
+        if out is None:
+            out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
+        _check("decode_attention", lib().decode_attention(self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens),
+                                                          n, _ptr(out), _stream(stream)))
+        return out
+
+    def score_steps(self, hidden, boundary_mask, row_trace, weights, step_scores_out=None, stream=None):
+        M = hidden.shape[0]
+        if step_scores_out is None:
+            step_scores_out = torch.empty(M, dtype=torch.float32, device=hidden.device)
+        _check("score_steps", lib().score_steps(self.handle, _ptr(hidden), _ptr(boundary_mask), _ptr(row_trace), M,
+                                                C.byref(weights.struct), _ptr(step_scores_out), _stream(stream)))
+        return step_scores_out
+
+    def prune_if_saturated(self, scores, threshold, keep_frac, stream=None):
+        """Returns (pruned_ids, n_pruned) device tensors owned by the pool (no sync)."""
+        _check("prune_if_saturated", lib().prune_if_saturated(self.handle, _ptr(scores), threshold, keep_frac,
+                                                              _ptr(self.pruned_ids), _ptr(self.n_pruned), _stream(stream)))
+        return self.pruned_ids, self.n_pruned
+
+    def release_traces(self, trace_ids, stream=None):
+        _check("kv_pool_release_traces", lib().kv_pool_release_traces(self.handle, _ptr(trace_ids), trace_ids.numel(),
+                                                                      _stream(stream)))
+
+    def stats(self, stream=None):
+        u, f, t, l = C.c_int(), C.c_int(), C.c_int(), C.c_int()
+        _check("kv_pool_stats", lib().kv_pool_stats(self.handle, C.byref(u), C.byref(f), C.byref(t), C.byref(l), _stream(stream)))
+        return dict(used=u.value, free=f.value, total=t.value, live_traces=l.value)
+
+    def last_error(self, stream=None):
+        mask = C.c_uint()
+        code = lib().kv_pool_last_error(self.handle, C.byref(mask), _stream(stream))
+        return code, mask.value
+
+    def read_kv(self, layer, kv_head, block_row, seq_len, stream=None):
+        k = torch.empty((seq_len, self.head_dim), dtype=self.torch_dtype, device=self.device)
+        v = torch.empty_like(k)
+        _check("kv_pool_read_kv", lib().kv_pool_read_kv(self.handle, layer, kv_head, _ptr(block_row), seq_len, _ptr(k),
+                                                        _ptr(v), _stream(stream)))
+        return k, v
+
+    def set_attention_config(self, grid_ctas=0, fast_path=0):
+        _check("kv_pool_set_attention_config", lib().kv_pool_set_attention_config(self.handle, grid_ctas, fast_path))
+
+
+class ScorerWeights:
+    """Device tensors of the step scorer plus the C struct that points at them."""
+
+    def __init__(self, W1, b1, w2, b2, dtype):
+        self.W1, self.b1, self.w2, self.b2 = W1.contiguous(), b1.contiguous(), w2.contiguous(), float(b2)
+        m, D = self.W1.shape
+        self.struct = scorer_weights(W1=self.W1.data_ptr(), b1=self.b1.data_ptr(), w2=self.w2.data_ptr(),
+                                     b2=self.b2, D=D, m=m, dtype=dtype)

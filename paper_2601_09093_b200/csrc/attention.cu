@@ -1,0 +1,585 @@
+// decode_attention: grouped-query decode attention over the paged KV pool.
+//
+//   out[i][h] = sum_j softmax_j(q[i][h] . K_i[j] / sqrt(d)) V_i[j]      (the attention inside
+// NextToken of Algorithm 1; decoding is where Table 3 / Fig. 2c put the non-waiting time).
+//
+// Two implementations:
+//  * attn_scalar_kernel - any dtype / head_dim / page size, one CTA per (trace, query head).
+//    Used for fp32 pools and for shapes the tensor-core kernel does not cover.
+//  * attn_mma_kernel - bf16, head_dim 128, page 16, G <= 16.  HBM-bound design:
+//      - the whole launch's KV stream (for every trace, for every KV head, its pages in order)
+//        is cut into gridDim * kWarps equal contiguous partitions; a warp owns one partition,
+//        so all SMs finish together whatever the mix of trace lengths, and no atomics or
+//        inter-CTA waits exist;
+//      - a page of one KV head (K 4 KiB + V 4 KiB, contiguous, pre-swizzled in HBM) is brought
+//        into shared memory by ONE bulk async copy that signals an mbarrier; every warp keeps
+//        its own ring of kStages pages in flight and never synchronises with another warp;
+//      - all G query heads of the group are served from that single read of K and V:
+//        S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the
+//        heads on the M axis, ldmatrix (plain for K, transposed for V) feeding the B operand;
+//      - running (max, sum) softmax state per head in fp32, exp2 with the scale folded in;
+//      - a partition that holds a whole (trace, head) sequence writes the output directly;
+//        otherwise it writes an (m, l, o) partial (at most two per warp) and attn_merge_kernel
+//        combines the partials of each split (trace, head).
+#include "step_internal.cuh"
+
+#include <math.h>
+
+using namespace stepk;
+
+namespace {
+
+// =============================================================== scalar kernel
+template <typename T> __device__ inline float ld_f32(const T* p);
+template <> __device__ inline float ld_f32<float>(const float* p) { return *p; }
+template <> __device__ inline float ld_f32<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+constexpr int kScalarWarps = 4;
+constexpr int kMaxDimsPerLane = 16;   // head_dim <= 512
+
+template <typename T>
+__global__ void __launch_bounds__(kScalarWarps * 32)
+attn_scalar_kernel(Geo g, const T* __restrict__ kv, int layer, const T* __restrict__ q,
+                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
+                   float* __restrict__ out, int32_t* counters) {
+  extern __shared__ float smf[];
+  float* s_q = smf;                                  // [d]
+  float* s_o = smf + g.d;                            // [warps][d]
+  __shared__ float s_m[kScalarWarps], s_l[kScalarWarps];
+  const int h = blockIdx.x, t = blockIdx.y, kvh = h / g.G;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cpe = 16 / (int)sizeof(T);
+  int S = seq_lens[t];
+  if (S < 0) S = 0;
+  if ((long long)S > (long long)g.max_pages * g.P) { S = g.max_pages * g.P; if (threadIdx.x == 0) flag_error(counters, STEP_ERR_CAPACITY); }
+  for (int k = threadIdx.x; k < g.d; k += blockDim.x) s_q[k] = ld_f32(q + ((size_t)t * g.Hq + h) * g.d + k);
+  __syncthreads();
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
+  float m = -INFINITY, l = 0.f;
+  float acc[kMaxDimsPerLane];
+#pragma unroll
+  for (int i = 0; i < kMaxDimsPerLane; ++i) acc[i] = 0.f;
+  for (int j = warp; j < S; j += kScalarWarps) {
+    const int page = j / g.P, slot = j % g.P;
+    int b = block_table[(size_t)t * g.max_pages + page];
+    if (b < 0 || b >= g.num_blocks) { if (lane == 0) flag_error(counters, STEP_ERR_BAD_BLOCK); b = 0; }
+    const T* kp = kv + kv_page_base(g, layer, b, kvh, 0);
+    const T* vp = kp + (size_t)g.P * g.d;
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < kMaxDimsPerLane; ++i) {
+      const int k = lane + 32 * i;
+      if (k < g.d) dot += s_q[k] * ld_f32(kp + kv_in_page(g, slot, k, cpe));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    const float s = dot * scale_log2;
+    const float m_new = fmaxf(m, s);
+    const float corr = exp2f(m - m_new), p = exp2f(s - m_new);
+    l = l * corr + p;
+#pragma unroll
+    for (int i = 0; i < kMaxDimsPerLane; ++i) {
+      const int k = lane + 32 * i;
+      if (k < g.d) acc[i] = acc[i] * corr + p * ld_f32(vp + kv_in_page(g, slot, k, cpe));
+    }
+    m = m_new;
+  }
+  if (lane == 0) { s_m[warp] = m; s_l[warp] = l; }
+#pragma unroll
+  for (int i = 0; i < kMaxDimsPerLane; ++i) {
+    const int k = lane + 32 * i;
+    if (k < g.d) s_o[warp * g.d + k] = acc[i];
+  }
+  __syncthreads();
+  float M = -INFINITY;
+  for (int w = 0; w < kScalarWarps; ++w) M = fmaxf(M, s_m[w]);
+  for (int k = threadIdx.x; k < g.d; k += blockDim.x) {
+    float num = 0.f, den = 0.f;
+    for (int w = 0; w < kScalarWarps; ++w) {
+      if (s_m[w] == -INFINITY) continue;           // that warp saw no position
+      const float wgt = exp2f(s_m[w] - M);
+      num += wgt * s_o[w * g.d + k];
+      den += wgt * s_l[w];
+    }
+    out[((size_t)t * g.Hq + h) * g.d + k] = den > 0.f ? num / den : 0.f;
+  }
+}
+
+// =============================================================== tensor-core kernel
+constexpr int kP = 16, kD = 128;
+constexpr int kPageBytes = 2 * kP * kD * 2;        // K rows then V rows of one KV head: 8 KiB
+constexpr int kVOffset = kP * kD * 2;              // 4 KiB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a bounded wait gives up after 2 s
+
+struct AttnArgs {
+  const __nv_bfloat16* kv_layer;   // kv_storage + layer offset
+  const __nv_bfloat16* q;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  float* out;
+  float* ws_ml;                    // [partition][2][G][2]
+  float* ws_o;                     // [partition][2][G][kD]
+  int32_t* counters;
+  int n, Hq, Hkv, G, max_pages, num_blocks;
+  float scale_log2;
+};
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ inline unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase with the given parity; false if the time limit ran out.
+__device__ inline bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+// One page: global (16-byte aligned) -> shared, completion counted in bytes on the mbarrier.
+__device__ inline void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ inline void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ inline void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ inline void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ inline uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Position in the launch's KV stream -> (trace, kv head, page).  The stream lists, for every
+// trace in order, for every KV head in order, that trace's pages in order.
+struct Cursor {
+  int t, h, page, np;   // np = pages of trace t
+};
+__device__ inline void cursor_seek(Cursor& c, const int* cum, int n, int Hkv, long long pos) {
+  int lo = 0, hi = n - 1;                              // largest t with Hkv * cum[t] <= pos
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
+  }
+  c.t = lo;
+  c.np = cum[lo + 1] - cum[lo];
+  const long long r = pos - (long long)Hkv * cum[lo];
+  c.h = (int)(r / c.np);
+  c.page = (int)(r % c.np);
+}
+__device__ inline void cursor_next(Cursor& c, const int* cum, int n, int Hkv) {
+  if (++c.page < c.np) return;
+  c.page = 0;
+  if (++c.h < Hkv) return;
+  c.h = 0;
+  do { ++c.t; } while (c.t < n && cum[c.t + 1] == cum[c.t]);
+  c.np = c.t < n ? cum[c.t + 1] - cum[c.t] : 1;
+}
+
+template <int kWarps, int kStages, bool kRows16>
+__global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* s_pages = smem;                                              // [kWarps][kStages][8 KiB]
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kWarps * kStages * kPageBytes);
+  int* s_cum = reinterpret_cast<int*>(s_bar + kWarps * kStages);              // [n + 1]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = a.n, Hkv = a.Hkv, G = a.G;
+
+  // ---- pages per trace, exclusive prefix sum (warp 0), barrier init (lane 0 of each warp)
+  if (warp == 0) {
+    int running = 0;
+    for (int base = 0; base < n; base += 32) {
+      const int t = base + lane;
+      int pages = 0;
+      if (t < n) {
+        int S = a.seq_lens[t];
+        if (S < 0) S = 0;
+        pages = (S + kP - 1) / kP;
+        if (pages > a.max_pages) { pages = a.max_pages; flag_error(a.counters, STEP_ERR_CAPACITY); }
+      }
+      int incl = pages;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (t < n) s_cum[t] = running + incl - pages;
+      running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_cum[n] = running;
+  }
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&s_bar[warp * kStages + s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  const long long total = (long long)Hkv * s_cum[n];
+  const int n_part = gridDim.x * kWarps;
+  const long long W = (total + n_part - 1) / n_part;
+  const int part = blockIdx.x * kWarps + warp;
+  const long long pos0 = (long long)part * W;
+  if (W == 0 || pos0 >= total) return;
+  const int cnt = (int)((pos0 + W <= total ? pos0 + W : total) - pos0);
+
+  unsigned char* my_pages = s_pages + (size_t)warp * kStages * kPageBytes;
+  const uint32_t my_pages_u32 = smem_u32(my_pages);
+  const uint32_t my_bar_u32 = smem_u32(&s_bar[warp * kStages]);
+
+  // ---- producer side: cursor, block-id window (lane i holds the id of page win_base + i)
+  Cursor pc;
+  cursor_seek(pc, s_cum, n, Hkv, pos0);
+  int win_t = -1, win_base = 0, win_ids = 0;
+  int issued = 0;
+  auto produce = [&](int stage) {
+    if (pc.t != win_t || pc.page < win_base || pc.page >= win_base + 32) {
+      win_t = pc.t; win_base = pc.page;
+      const int pg = win_base + lane;
+      win_ids = pg < pc.np ? a.block_table[(size_t)pc.t * a.max_pages + pg] : 0;
+    }
+    int b = __shfl_sync(0xffffffffu, win_ids, pc.page - win_base);
+    if (lane == 0) {
+      if (b < 0 || b >= a.num_blocks) { flag_error(a.counters, STEP_ERR_BAD_BLOCK); b = 0; }
+      const __nv_bfloat16* src = a.kv_layer + ((size_t)b * Hkv + pc.h) * (size_t)(2 * kP * kD);
+      const uint32_t bar = my_bar_u32 + stage * 8;
+      mbar_expect_tx(bar, kPageBytes);
+      bulk_load(my_pages_u32 + stage * kPageBytes, src, kPageBytes, bar);
+    }
+    cursor_next(pc, s_cum, n, Hkv);
+    ++issued;
+  };
+  for (int s = 0; s < kStages && issued < cnt; ++s) produce(s);
+
+  // ---- consumer side
+  Cursor cc;
+  cursor_seek(cc, s_cum, n, Hkv, pos0);
+  const int g_row = lane >> 2, tq = lane & 3;
+  uint32_t qa[8][4];                 // A fragments of Q for the 8 k-steps over head_dim
+  float o_acc[16][4];                // O fragments: 16 n-tiles over head_dim
+  float m_run[2], l_run[2];          // rows g_row and g_row + 8
+  int seg_first_page = 0;
+  bool seg_open = false, seg_is_first = true;
+  int stage = 0;
+  uint32_t parity = 0;
+  bool alive = true;
+
+  // ldmatrix lane addressing inside a page (swizzled 16-byte chunks: chunk' = chunk ^ (row & 7))
+  const int mi = lane >> 3, r8 = lane & 7;
+  const int k_row = ((mi >> 1) << 3) + r8;             // K: matrices 0,1 -> tokens 0-7; 2,3 -> tokens 8-15
+  const int k_csel = mi & 1;                           //    matrix parity picks the low/high 8 dims of the k-step
+  const int v_row = ((mi & 1) << 3) + r8;              // V: matrices 0,2 -> tokens 0-7; 1,3 -> tokens 8-15
+  const int v_csel = mi >> 1;                          //    matrices 2,3 belong to the next 8-wide dim tile
+
+  for (int i = 0; i < cnt; ++i) {
+    if (!seg_open) {
+      // new (trace, head) segment: Q fragments of the G heads of this group, fresh softmax state
+      const __nv_bfloat16* qbase = a.q + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
+      const uint32_t* q0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)g_row * kD);
+      const uint32_t* q1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(g_row + 8) * kD);
+      const bool r0 = g_row < G, r1 = kRows16 && (g_row + 8 < G);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qa[ks][0] = r0 ? q0[ks * 8 + tq] : 0u;
+        qa[ks][2] = r0 ? q0[ks * 8 + 4 + tq] : 0u;
+        qa[ks][1] = r1 ? q1[ks * 8 + tq] : 0u;
+        qa[ks][3] = r1 ? q1[ks * 8 + 4 + tq] : 0u;
+      }
+#pragma unroll
+      for (int dt = 0; dt < 16; ++dt) { o_acc[dt][0] = o_acc[dt][1] = o_acc[dt][2] = o_acc[dt][3] = 0.f; }
+      m_run[0] = m_run[1] = -INFINITY;
+      l_run[0] = l_run[1] = 0.f;
+      seg_first_page = cc.page;
+      seg_open = true;
+    }
+
+    if (!mbar_wait_bounded(my_bar_u32 + stage * 8, parity)) {
+      if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
+      alive = false;
+      break;
+    }
+    const uint32_t kpage = my_pages_u32 + stage * kPageBytes;
+    const uint32_t vpage = kpage + kVOffset;
+
+    // tokens of this page that exist (only the last page of a sequence can be short)
+    int valid = kP;
+    if (cc.page == cc.np - 1) {
+      int S = a.seq_lens[cc.t];
+      const int cap = a.max_pages * kP;
+      if (S > cap) S = cap;
+      valid = S - cc.page * kP;
+      if (valid < kP) {
+        // unused V rows may hold anything (even NaN bit patterns): zero them so 0 * V stays 0
+        for (int idx = lane; idx < (kP - valid) * 16; idx += 32) {
+          const int row = valid + (idx >> 4), chunk = idx & 15;
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vpage + row * 256 + chunk * 16), "r"(0u) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+      }
+    }
+
+    // ---- S = Q K^T for 16 tokens: two n-tiles of 8 tokens
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      const int chunk = ks * 2 + k_csel;
+      const uint32_t addr = kpage + k_row * 256 + ((((chunk & 8) | ((chunk ^ k_row) & 7))) << 4);
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4(addr, b0, b1, b2, b3);
+      mma_bf16(s0, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+      mma_bf16(s1, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+    }
+    // thread holds, for row g_row (and g_row+8): tokens 2tq, 2tq+1 (s0) and 8+2tq, 9+2tq (s1)
+    {
+      const int j0 = 2 * tq;
+      const bool v00 = j0 < valid, v01 = j0 + 1 < valid, v10 = j0 + 8 < valid, v11 = j0 + 9 < valid;
+      s0[0] = v00 ? s0[0] * a.scale_log2 : -INFINITY; s0[1] = v01 ? s0[1] * a.scale_log2 : -INFINITY;
+      s1[0] = v10 ? s1[0] * a.scale_log2 : -INFINITY; s1[1] = v11 ? s1[1] * a.scale_log2 : -INFINITY;
+      if (kRows16) {
+        s0[2] = v00 ? s0[2] * a.scale_log2 : -INFINITY; s0[3] = v01 ? s0[3] * a.scale_log2 : -INFINITY;
+        s1[2] = v10 ? s1[2] * a.scale_log2 : -INFINITY; s1[3] = v11 ? s1[3] * a.scale_log2 : -INFINITY;
+      }
+    }
+    float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    const float mn0 = fmaxf(m_run[0], mx0);          // finite: token 0 of a page always exists
+    const float corr0 = exp2f(m_run[0] - mn0);
+    m_run[0] = mn0;
+    const float p00 = exp2f(s0[0] - mn0), p01 = exp2f(s0[1] - mn0), p10 = exp2f(s1[0] - mn0), p11 = exp2f(s1[1] - mn0);
+    l_run[0] = l_run[0] * corr0 + (p00 + p01) + (p10 + p11);
+    uint32_t pa0 = pack_bf16(p00, p01), pa2 = pack_bf16(p10, p11), pa1 = 0u, pa3 = 0u;
+    float corr1 = 1.f;
+    if (kRows16) {
+      float mx1 = fmaxf(fmaxf(s0[2], s0[3]), fmaxf(s1[2], s1[3]));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn1 = fmaxf(m_run[1], mx1);
+      corr1 = exp2f(m_run[1] - mn1);
+      m_run[1] = mn1;
+      const float q00 = exp2f(s0[2] - mn1), q01 = exp2f(s0[3] - mn1), q10 = exp2f(s1[2] - mn1), q11 = exp2f(s1[3] - mn1);
+      l_run[1] = l_run[1] * corr1 + (q00 + q01) + (q10 + q11);
+      pa1 = pack_bf16(q00, q01); pa3 = pack_bf16(q10, q11);
+    }
+    // rescale O only when some row's maximum moved (warp-uniform branch)
+    const bool moved = (corr0 != 1.f) || (kRows16 && corr1 != 1.f);
+    if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll
+      for (int dt = 0; dt < 16; ++dt) {
+        o_acc[dt][0] *= corr0; o_acc[dt][1] *= corr0;
+        if (kRows16) { o_acc[dt][2] *= corr1; o_acc[dt][3] *= corr1; }
+      }
+    }
+    // ---- O += P V : 16 n-tiles over head_dim, k = 16 tokens
+#pragma unroll
+    for (int dp = 0; dp < 8; ++dp) {
+      const int chunk = dp * 2 + v_csel;
+      const uint32_t addr = vpage + v_row * 256 + ((((chunk & 8) | ((chunk ^ v_row) & 7))) << 4);
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4_t(addr, b0, b1, b2, b3);
+      mma_bf16(o_acc[2 * dp], pa0, pa1, pa2, pa3, b0, b1);
+      mma_bf16(o_acc[2 * dp + 1], pa0, pa1, pa2, pa3, b2, b3);
+    }
+    __syncwarp();
+    if (issued < cnt) produce(stage);                  // refill the stage just consumed
+
+    // ---- end of this (trace, head) segment?
+    const bool seg_end = (cc.page + 1 == cc.np) || (i + 1 == cnt);
+    if (seg_end) {
+      float l0 = l_run[0];
+      l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+      l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+      float l1 = l_run[1];
+      if (kRows16) {
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+      }
+      const bool complete = seg_first_page == 0 && cc.page + 1 == cc.np;
+      if (complete) {
+        float* ob = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
+        if (g_row < G) {
+          const float inv = 1.f / l0;
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(ob + (size_t)g_row * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][0] * inv, o_acc[dt][1] * inv);
+        }
+        if (kRows16 && g_row + 8 < G) {
+          const float inv = 1.f / l1;
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2] * inv, o_acc[dt][3] * inv);
+        }
+      } else {
+        const size_t slot = (size_t)part * 2 + (seg_is_first ? 0 : 1);
+        float* ml = a.ws_ml + slot * G * 2;
+        float* ob = a.ws_o + slot * G * kD;
+        if (g_row < G) {
+          if (tq == 0) { ml[g_row * 2] = m_run[0]; ml[g_row * 2 + 1] = l0; }
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(ob + (size_t)g_row * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][0], o_acc[dt][1]);
+        }
+        if (kRows16 && g_row + 8 < G) {
+          if (tq == 0) { ml[(g_row + 8) * 2] = m_run[1]; ml[(g_row + 8) * 2 + 1] = l1; }
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2], o_acc[dt][3]);
+        }
+      }
+      seg_open = false;
+      seg_is_first = false;
+    }
+    cursor_next(cc, s_cum, n, Hkv);
+    if (++stage == kStages) { stage = 0; parity ^= 1; }
+  }
+
+  if (!alive) {
+    // A wait ran out.  Copies already issued still target this CTA's shared memory, so give each
+    // of them one more bounded wait before the warp leaves; nothing else is touched.
+    for (int s = 0; s < kStages; ++s) {
+      mbar_wait_bounded(my_bar_u32 + s * 8, 0);
+      mbar_wait_bounded(my_bar_u32 + s * 8, 1);
+    }
+  }
+}
+
+// Combines the partials of every (trace, kv head) sequence that more than one partition touched,
+// and writes zeros for empty sequences.  grid (Hkv, n), kD threads.
+__global__ void __launch_bounds__(kD) attn_merge_kernel(AttnArgs a, int n_part) {
+  __shared__ int s_red[2][kD / 32];
+  const int h = blockIdx.x, t = blockIdx.y, n = a.n, G = a.G;
+  int before = 0, all = 0, mine = 0;
+  for (int u = threadIdx.x; u < n; u += blockDim.x) {
+    int S = a.seq_lens[u];
+    if (S < 0) S = 0;
+    int pages = (S + kP - 1) / kP;
+    if (pages > a.max_pages) pages = a.max_pages;
+    all += pages;
+    if (u < t) before += pages;
+    if (u == t) mine = pages;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    all += __shfl_xor_sync(0xffffffffu, all, o);
+    mine += __shfl_xor_sync(0xffffffffu, mine, o);
+  }
+  __shared__ int s_mine[kD / 32];
+  if ((threadIdx.x & 31) == 0) { s_red[0][threadIdx.x >> 5] = before; s_red[1][threadIdx.x >> 5] = all; s_mine[threadIdx.x >> 5] = mine; }
+  __syncthreads();
+  before = all = mine = 0;
+  for (int w = 0; w < kD / 32; ++w) { before += s_red[0][w]; all += s_red[1][w]; mine += s_mine[w]; }
+  const int np = mine;
+  float* ob = a.out + ((size_t)t * a.Hq + (size_t)h * G) * kD;
+  if (np == 0) {
+    for (int g = 0; g < G; ++g) ob[(size_t)g * kD + threadIdx.x] = 0.f;
+    return;
+  }
+  const long long total = (long long)a.Hkv * all;
+  const long long W = (total + n_part - 1) / n_part;
+  const long long start = (long long)a.Hkv * before + (long long)h * np;
+  const int w_first = (int)(start / W), w_last = (int)((start + np - 1) / W);
+  if (w_first == w_last) return;                       // written whole by one warp
+  for (int g = 0; g < G; ++g) {
+    float M = -INFINITY;
+    for (int w = w_first; w <= w_last; ++w) {
+      const size_t slot = (size_t)w * 2 + (start <= (long long)w * W ? 0 : 1);
+      M = fmaxf(M, a.ws_ml[(slot * G + g) * 2]);
+    }
+    float num = 0.f, den = 0.f;
+    for (int w = w_first; w <= w_last; ++w) {
+      const size_t slot = (size_t)w * 2 + (start <= (long long)w * W ? 0 : 1);
+      const float wgt = exp2f(a.ws_ml[(slot * G + g) * 2] - M);
+      den += wgt * a.ws_ml[(slot * G + g) * 2 + 1];
+      num += wgt * a.ws_o[(slot * G + g) * kD + threadIdx.x];
+    }
+    ob[(size_t)g * kD + threadIdx.x] = num / den;
+  }
+}
+
+constexpr int kWarpsDefault = 8, kStagesDefault = 3;
+
+template <int kWarps, int kStages>
+int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s) {
+  const size_t smem = (size_t)kWarps * kStages * kPageBytes + (size_t)kWarps * kStages * 8 + (size_t)(a.n + 1) * 4;
+  int grid = pool->attn_grid;
+  if (grid * kWarps > kMaxPartitions) grid = kMaxPartitions / kWarps;
+  if (grid < 1) grid = 1;
+  if (a.G > 8) {
+    auto kern = attn_mma_kernel<kWarps, kStages, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+    kern<<<grid, kWarps * 32, smem, s>>>(a);
+  } else {
+    auto kern = attn_mma_kernel<kWarps, kStages, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+    kern<<<grid, kWarps * 32, smem, s>>>(a);
+  }
+  attn_merge_kernel<<<dim3(a.Hkv, a.n), kD, 0, s>>>(a, grid * kWarps);
+  return launch_ok();
+}
+
+}  // namespace
+
+extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                const int32_t* seq_lens, int n, void* out, void* stream) {
+  if (!pool || n < 0) return STEP_ERR_INVALID_ARG;
+  if (n == 0) return STEP_OK;
+  if (!q || !block_table || !seq_lens || !out) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  if (layer < 0 || layer >= g.L) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool fast = pool->fast_path > 0 && pool->cfg.dtype == STEP_BF16 && g.d == kD && g.P == kP &&
+                    g.G <= 16 && n <= kMaxTracesFast && pool->swizzle;
+  if (fast) {
+    AttnArgs a;
+    a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
+    a.q = (const __nv_bfloat16*)q;
+    a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
+    a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.counters = pool->v.counters;
+    a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
+    return launch_mma<kWarpsDefault, kStagesDefault>(pool, a, s);
+  }
+  if (n > 65535) return STEP_ERR_INVALID_ARG;
+  const size_t smem = (size_t)(g.d + kScalarWarps * g.d) * sizeof(float);
+  if (pool->cfg.dtype == STEP_BF16)
+    attn_scalar_kernel<__nv_bfloat16><<<dim3(g.Hq, n), kScalarWarps * 32, smem, s>>>(
+        g, (const __nv_bfloat16*)pool->cfg.kv_storage, layer, (const __nv_bfloat16*)q, block_table, seq_lens,
+        (float*)out, pool->v.counters);
+  else
+    attn_scalar_kernel<float><<<dim3(g.Hq, n), kScalarWarps * 32, smem, s>>>(
+        g, (const float*)pool->cfg.kv_storage, layer, (const float*)q, block_table, seq_lens, (float*)out,
+        pool->v.counters);
+  return launch_ok();
+}

@@ -1,0 +1,441 @@
+// Paged KV pool: creation, InitTraces prefix fork, append_kv, accessors.
+// (Algorithm 1: InitTraces and the cache write of NextToken; block bookkeeping is the
+// library's own since the paper delegates it to its inference engine.)
+#include "step_internal.cuh"
+
+#include <new>
+#include <vector>
+
+using namespace stepk;
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool config_valid(const kv_pool_config* c) {
+  if (!c) return false;
+  if (c->num_layers < 1 || c->num_q_heads < 1 || c->num_kv_heads < 1 || c->head_dim < 1) return false;
+  if (c->page_size < 1 || c->num_blocks < 1 || c->max_traces < 1 || c->max_pages_per_trace < 1) return false;
+  if (c->num_q_heads % c->num_kv_heads != 0) return false;
+  if (c->num_q_heads / c->num_kv_heads > 16) return false;
+  if (c->dtype != STEP_BF16 && c->dtype != STEP_FP32) return false;
+  int eb = c->dtype == STEP_BF16 ? 2 : 4;
+  if ((c->head_dim * eb) % 16 != 0 || c->head_dim > 512) return false;   // rows move as 16-byte chunks
+  if (c->max_score_rows < 0) return false;
+  if ((long long)c->max_traces * c->max_pages_per_trace > (1ll << 31) - 1) return false;
+  return true;
+}
+
+MetaLayout make_layout(const kv_pool_config* c) {
+  MetaLayout l;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t T = c->max_traces, NB = c->num_blocks;
+  const size_t rows = c->max_score_rows > 0 ? c->max_score_rows : c->max_traces;
+  const int G = c->num_q_heads / c->num_kv_heads;
+  l.block_table = take(T * c->max_pages_per_trace * 4);
+  l.seq_lens = take(T * 4);
+  l.live = take(T);
+  l.score_sum = take(T * 4);
+  l.score_cnt = take(T * 4);
+  l.trace_scores = take(T * 4);
+  l.refcount = take(NB * 4);
+  l.free_list = take(NB * 4);
+  l.claim = take(NB * 4);
+  l.counters = take(C_NUM * 4);
+  l.append_base = take(T * 4);
+  l.prune_rank = take(T * 4);
+  l.prune_list = take(T * 4);
+  l.prune_off = take((T + 1) * 4);
+  l.score_idx = take(rows * 4);
+  l.score_z = take(rows * kScoreSplits * 4);
+  l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
+  l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
+  l.total = off;
+  return l;
+}
+
+size_t kv_bytes_of(const kv_pool_config* c) {
+  size_t eb = c->dtype == STEP_BF16 ? 2 : 4;
+  return (size_t)c->num_layers * c->num_blocks * c->num_kv_heads * 2 * c->page_size * c->head_dim * eb;
+}
+
+__global__ void init_meta_kernel(DevViews v, Geo g, float unscored) {
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const size_t nbt = (size_t)g.max_traces * g.max_pages;
+  for (size_t i = tid; i < nbt; i += stride) v.block_table[i] = -1;
+  for (size_t i = tid; i < (size_t)g.max_traces; i += stride) {
+    v.seq_lens[i] = 0; v.live[i] = 0; v.score_sum[i] = 0.f; v.score_cnt[i] = 0;
+    v.trace_scores[i] = unscored; v.append_base[i] = -1;
+  }
+  for (size_t i = tid; i < (size_t)g.num_blocks; i += stride) {
+    v.refcount[i] = 0; v.claim[i] = -1;
+    v.free_list[i] = g.num_blocks - 1 - (int)i;       // a stack: the first pop is block 0
+  }
+  for (size_t i = tid; i < (size_t)C_NUM; i += stride) v.counters[i] = (i == C_FREE_COUNT) ? g.num_blocks : 0;
+}
+
+// ---------------------------------------------------------------- InitTraces (fork)
+__global__ void fork_alloc_kernel(DevViews v, Geo g, int first_trace, int n_traces, int prefix_len) {
+  __shared__ int s_ok, s_fc;
+  const int full = prefix_len / g.P, rem = prefix_len % g.P;
+  const int needed = full + (rem ? n_traces : 0);
+  if (threadIdx.x == 0) {
+    s_fc = v.counters[C_FREE_COUNT];
+    s_ok = needed <= s_fc;
+    v.counters[C_FORK_OK] = s_ok;
+    if (!s_ok) flag_error(v.counters, STEP_ERR_NO_BLOCKS);
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  const int fc = s_fc;
+  // shared full pages: pop in page order
+  for (int p = threadIdx.x; p < full; p += blockDim.x) v.refcount[v.free_list[fc - 1 - p]] = n_traces;
+  for (int j = 0; j < n_traces; ++j) {
+    int32_t* row = v.block_table + (size_t)(first_trace + j) * g.max_pages;
+    for (int p = threadIdx.x; p < full; p += blockDim.x) row[p] = v.free_list[fc - 1 - p];
+  }
+  // private copy of the partial last page, one block per trace in trace order
+  for (int j = threadIdx.x; j < n_traces; j += blockDim.x) {
+    const int t = first_trace + j;
+    if (rem) {
+      int b = v.free_list[fc - 1 - full - j];
+      v.refcount[b] = 1;
+      v.block_table[(size_t)t * g.max_pages + full] = b;
+    }
+    v.seq_lens[t] = prefix_len;
+    v.live[t] = 1;
+    v.score_sum[t] = 0.f; v.score_cnt[t] = 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) v.counters[C_FREE_COUNT] = fc - needed;
+}
+
+// One thread moves one 16-byte chunk of the prompt's K or V.
+__global__ void fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ kpre,
+                                  const uint4* __restrict__ vpre, int first_trace, int n_traces,
+                                  int prefix_len, int cpr /*chunks per row*/, int cpe) {
+  if (!v.counters[C_FORK_OK]) return;
+  const int full = prefix_len / g.P;
+  const size_t per_kv = (size_t)g.L * g.Hkv * prefix_len * cpr;
+  const size_t total = per_kv * 2;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int which = i >= per_kv;
+    size_t r = which ? i - per_kv : i;
+    const int c = r % cpr; r /= cpr;
+    const int pos = r % prefix_len; r /= prefix_len;
+    const int head = r % g.Hkv; const int layer = r / g.Hkv;
+    const uint4 val = (which ? vpre : kpre)[i - (which ? per_kv : 0)];
+    const int page = pos / g.P, slot = pos % g.P;
+    const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
+    const int copies = page < full ? 1 : n_traces;     // the partial page is private per trace
+    for (int j = 0; j < copies; ++j) {
+      const int b = v.block_table[(size_t)(first_trace + j) * g.max_pages + page];
+      const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
+      kv[e / cpe + cdst] = val;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- append_kv
+// Phase 1 (one CTA): decide, in list order, which traces get their pages; pop blocks.
+__global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, int n_tokens) {
+  extern __shared__ int sm[];
+  int* s_need = sm;            // pages wanted, or -1 if the trace is skipped
+  int* s_off = sm + n;         // pops that precede this trace's
+  int* s_have = sm + 2 * n;
+  __shared__ int s_fc;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int t = ids[i];
+    int need = -1, have = 0;
+    if (t < 0 || t >= g.max_traces || !v.live[t]) {
+      flag_error(v.counters, STEP_ERR_BAD_TRACE);
+    } else {
+      const int S = v.seq_lens[t];
+      have = (S + g.P - 1) / g.P;
+      const long long want = ((long long)S + n_tokens + g.P - 1) / g.P;
+      if (want > g.max_pages) flag_error(v.counters, STEP_ERR_CAPACITY);
+      else need = (int)want - have;
+    }
+    s_need[i] = need; s_have[i] = have;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int fc = v.counters[C_FREE_COUNT];
+    int remaining = fc;
+    for (int i = 0; i < n; ++i) {
+      const int need = s_need[i];
+      if (need < 0) continue;
+      if (need > remaining) { s_need[i] = -1; flag_error(v.counters, STEP_ERR_NO_BLOCKS); continue; }
+      s_off[i] = fc - remaining;
+      remaining -= need;
+    }
+    s_fc = fc;
+    v.counters[C_FREE_COUNT] = remaining;
+  }
+  __syncthreads();
+  const int fc = s_fc;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  for (int i = warp; i < n; i += nwarps) {
+    const int need = s_need[i];
+    const int t = ids[i];
+    if (need < 0) { if (lane == 0) v.append_base[i] = -1; continue; }
+    int32_t* row = v.block_table + (size_t)t * g.max_pages;
+    for (int p = lane; p < need; p += 32) {
+      const int b = v.free_list[fc - 1 - s_off[i] - p];
+      row[s_have[i] + p] = b;
+      v.refcount[b] = 1;
+    }
+    if (lane == 0) {
+      const int S = v.seq_lens[t];
+      v.append_base[i] = S;
+      v.seq_lens[t] = S + n_tokens;
+    }
+  }
+}
+
+// Phase 2: one thread moves one 16-byte chunk of a new K or V row into its page.
+__global__ void append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ knew,
+                                    const uint4* __restrict__ vnew, const int32_t* __restrict__ ids,
+                                    int n, int n_tokens, int cpr, int cpe) {
+  const size_t per_kv = (size_t)n * n_tokens * g.L * g.Hkv * cpr;
+  const size_t total = per_kv * 2;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int which = i >= per_kv;
+    const size_t src = which ? i - per_kv : i;
+    size_t r = src;
+    const int c = r % cpr; r /= cpr;
+    const int head = r % g.Hkv; r /= g.Hkv;
+    const int layer = r % g.L; r /= g.L;
+    const int j = r % n_tokens; const int idx = r / n_tokens;
+    const int base = v.append_base[idx];
+    if (base < 0) continue;
+    const int t = ids[idx];
+    const int pos = base + j, page = pos / g.P, slot = pos % g.P;
+    const int b = v.block_table[(size_t)t * g.max_pages + page];
+    const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
+    const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
+    kv[e / cpe + cdst] = (which ? vnew : knew)[src];
+  }
+}
+
+// ---------------------------------------------------------------- read-back of logical rows
+__global__ void read_kv_kernel(Geo g, const uint4* __restrict__ kv, int layer, int head,
+                               const int32_t* __restrict__ block_row, int seq_len, uint4* __restrict__ k_out,
+                               uint4* __restrict__ v_out, int cpr, int cpe, int32_t* counters) {
+  const size_t total = (size_t)seq_len * cpr * 2;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int which = i >= (size_t)seq_len * cpr;
+    size_t r = which ? i - (size_t)seq_len * cpr : i;
+    const int c = r % cpr; const int pos = r / cpr;
+    const int page = pos / g.P, slot = pos % g.P;
+    const int b = block_row[page];
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (b < 0 || b >= g.num_blocks) {
+      flag_error(counters, STEP_ERR_BAD_BLOCK);
+    } else {
+      const int csrc = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
+      const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
+      val = kv[e / cpe + csrc];
+    }
+    (which ? v_out : k_out)[(size_t)pos * cpr + c] = val;
+  }
+}
+
+int grid_for(size_t items, int threads, int num_sms) {
+  size_t blocks = (items + threads - 1) / threads;
+  size_t cap = (size_t)num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* step_version(void) { return "libstep 0.1 (sm_100a)"; }
+
+int kv_pool_required_bytes(const kv_pool_config* cfg, size_t* kv_bytes, size_t* meta_bytes) {
+  if (!config_valid(cfg)) return STEP_ERR_INVALID_ARG;
+  if (kv_bytes) *kv_bytes = kv_bytes_of(cfg);
+  if (meta_bytes) *meta_bytes = make_layout(cfg).total;
+  return STEP_OK;
+}
+
+int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
+  if (!out) return STEP_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_valid(cfg)) return STEP_ERR_INVALID_ARG;
+  if (!cfg->kv_storage || !cfg->meta_storage) return STEP_ERR_INVALID_ARG;
+  if (((uintptr_t)cfg->kv_storage | (uintptr_t)cfg->meta_storage) & 255) return STEP_ERR_INVALID_ARG;
+  MetaLayout lay = make_layout(cfg);
+  if (cfg->kv_bytes < kv_bytes_of(cfg) || cfg->meta_bytes < lay.total) return STEP_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  STEP_CUDA_OK(cudaGetDevice(&dev));
+  STEP_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  step_pool* p = new (std::nothrow) step_pool();
+  if (!p) return STEP_ERR_INVALID_ARG;
+  p->cfg = *cfg;
+  p->G = cfg->num_q_heads / cfg->num_kv_heads;
+  p->elem_bytes = cfg->dtype == STEP_BF16 ? 2 : 4;
+  p->swizzle = (cfg->dtype == STEP_BF16 && cfg->head_dim % 64 == 0) ? 1 : 0;
+  p->max_score_rows = cfg->max_score_rows > 0 ? cfg->max_score_rows : cfg->max_traces;
+  p->next_trace = 0;
+  p->num_sms = sms;
+  p->attn_grid = sms;
+  p->fast_path = 1;
+  p->device = dev;
+  p->lay = lay;
+  char* m = static_cast<char*>(cfg->meta_storage);
+  DevViews& v = p->v;
+  v.block_table = (int32_t*)(m + lay.block_table); v.seq_lens = (int32_t*)(m + lay.seq_lens);
+  v.live = (uint8_t*)(m + lay.live); v.score_sum = (float*)(m + lay.score_sum);
+  v.score_cnt = (int32_t*)(m + lay.score_cnt); v.trace_scores = (float*)(m + lay.trace_scores);
+  v.refcount = (int32_t*)(m + lay.refcount); v.free_list = (int32_t*)(m + lay.free_list);
+  v.claim = (int32_t*)(m + lay.claim); v.counters = (int32_t*)(m + lay.counters);
+  v.append_base = (int32_t*)(m + lay.append_base); v.prune_rank = (int32_t*)(m + lay.prune_rank);
+  v.prune_list = (int32_t*)(m + lay.prune_list); v.prune_off = (int32_t*)(m + lay.prune_off);
+  v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
+  v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o);
+  int st = kv_pool_reset(p, nullptr);
+  if (st == STEP_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = STEP_ERR_CUDA;
+  if (st != STEP_OK) { delete p; return st; }
+  *out = p;
+  return STEP_OK;
+}
+
+int kv_pool_destroy(step_pool* pool) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  delete pool;
+  return STEP_OK;
+}
+
+int kv_pool_reset(step_pool* pool, void* stream) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  size_t items = (size_t)g.max_traces * g.max_pages;
+  if ((size_t)g.num_blocks > items) items = g.num_blocks;
+  init_meta_kernel<<<grid_for(items, 256, pool->num_sms), 256, 0, (cudaStream_t)stream>>>(pool->v, g, pool->cfg.unscored_score);
+  pool->next_trace = 0;
+  return launch_ok();
+}
+
+int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const void* k_prefix,
+                        const void* v_prefix, int32_t* trace_ids_out, void* stream) {
+  if (!pool || n_traces < 1 || prefix_len < 0) return STEP_ERR_INVALID_ARG;
+  if (prefix_len > 0 && (!k_prefix || !v_prefix)) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  if (pool->next_trace + n_traces > g.max_traces) return STEP_ERR_CAPACITY;
+  if ((prefix_len + g.P - 1) / g.P > g.max_pages) return STEP_ERR_CAPACITY;
+  const int first = pool->next_trace;
+  cudaStream_t s = (cudaStream_t)stream;
+  fork_alloc_kernel<<<1, 256, 0, s>>>(pool->v, g, first, n_traces, prefix_len);
+  if (prefix_len > 0) {
+    const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
+    size_t chunks = (size_t)g.L * g.Hkv * prefix_len * cpr * 2;
+    fork_write_kernel<<<grid_for(chunks, 256, pool->num_sms), 256, 0, s>>>(
+        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_prefix, (const uint4*)v_prefix, first,
+        n_traces, prefix_len, cpr, cpe);
+  }
+  pool->next_trace += n_traces;
+  if (trace_ids_out) for (int j = 0; j < n_traces; ++j) trace_ids_out[j] = first + j;
+  return launch_ok();
+}
+
+int append_kv(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
+              const void* v_new, void* stream) {
+  if (!pool || n < 0 || n_tokens < 0) return STEP_ERR_INVALID_ARG;
+  if (n == 0 || n_tokens == 0) return STEP_OK;
+  if (!trace_ids || !k_new || !v_new) return STEP_ERR_INVALID_ARG;
+  if (n > pool->cfg.max_traces) return STEP_ERR_INVALID_ARG;   // ids must be distinct
+  Geo g = geo_of(pool);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
+  const size_t row_chunks = (size_t)n_tokens * g.L * g.Hkv * cpr;   // 16-byte chunks of K (or V) per trace
+  constexpr int kListChunk = 4096;                                  // traces per launch (shared-memory scan)
+  for (int off = 0; off < n; off += kListChunk) {
+    const int m = n - off < kListChunk ? n - off : kListChunk;
+    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens);
+    append_write_kernel<<<grid_for(row_chunks * m * 2, 256, pool->num_sms), 256, 0, s>>>(
+        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + row_chunks * off,
+        (const uint4*)v_new + row_chunks * off, trace_ids + off, m, n_tokens, cpr, cpe);
+  }
+  return launch_ok();
+}
+
+int kv_pool_stats(step_pool* pool, int* used, int* free_, int* total, int* live_traces, void* stream) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int fc = 0;
+  std::vector<uint8_t> live(pool->cfg.max_traces);
+  STEP_CUDA_OK(cudaMemcpyAsync(&fc, pool->v.counters + C_FREE_COUNT, sizeof(int), cudaMemcpyDeviceToHost, s));
+  STEP_CUDA_OK(cudaMemcpyAsync(live.data(), pool->v.live, live.size(), cudaMemcpyDeviceToHost, s));
+  STEP_CUDA_OK(cudaStreamSynchronize(s));
+  int nl = 0;
+  for (uint8_t b : live) nl += b != 0;
+  if (used) *used = pool->cfg.num_blocks - fc;
+  if (free_) *free_ = fc;
+  if (total) *total = pool->cfg.num_blocks;
+  if (live_traces) *live_traces = nl;
+  return STEP_OK;
+}
+
+int kv_pool_device_views(step_pool* pool, int32_t** block_table, int32_t** seq_lens, float** trace_scores,
+                         int32_t** free_list, int32_t** free_count, int32_t** refcount, uint8_t** live) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  if (block_table) *block_table = pool->v.block_table;
+  if (seq_lens) *seq_lens = pool->v.seq_lens;
+  if (trace_scores) *trace_scores = pool->v.trace_scores;
+  if (free_list) *free_list = pool->v.free_list;
+  if (free_count) *free_count = pool->v.counters + C_FREE_COUNT;
+  if (refcount) *refcount = pool->v.refcount;
+  if (live) *live = pool->v.live;
+  return STEP_OK;
+}
+
+int kv_pool_score_views(step_pool* pool, float** score_sum, int32_t** score_cnt) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  if (score_sum) *score_sum = pool->v.score_sum;
+  if (score_cnt) *score_cnt = pool->v.score_cnt;
+  return STEP_OK;
+}
+
+int kv_pool_last_error(step_pool* pool, unsigned* mask_out, void* stream) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned mask = 0;
+  STEP_CUDA_OK(cudaMemcpyAsync(&mask, pool->v.counters + C_STATUS, sizeof(mask), cudaMemcpyDeviceToHost, s));
+  STEP_CUDA_OK(cudaMemsetAsync(pool->v.counters + C_STATUS, 0, sizeof(int), s));
+  STEP_CUDA_OK(cudaStreamSynchronize(s));
+  if (mask_out) *mask_out = mask;
+  for (int code = 1; code < 32; ++code)
+    if (mask & (1u << code)) return code;
+  return STEP_OK;
+}
+
+int kv_pool_read_kv(step_pool* pool, int layer, int kv_head, const int32_t* block_row, int seq_len,
+                    void* k_out, void* v_out, void* stream) {
+  if (!pool || !block_row || seq_len < 0) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  if (layer < 0 || layer >= g.L || kv_head < 0 || kv_head >= g.Hkv) return STEP_ERR_INVALID_ARG;
+  if ((seq_len + g.P - 1) / g.P > g.max_pages) return STEP_ERR_INVALID_ARG;
+  if (seq_len == 0) return STEP_OK;
+  if (!k_out || !v_out) return STEP_ERR_INVALID_ARG;
+  const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
+  size_t chunks = (size_t)seq_len * cpr * 2;
+  read_kv_kernel<<<grid_for(chunks, 256, pool->num_sms), 256, 0, (cudaStream_t)stream>>>(
+      g, (const uint4*)pool->cfg.kv_storage, layer, kv_head, block_row, seq_len, (uint4*)k_out, (uint4*)v_out,
+      cpr, cpe, pool->v.counters);
+  return launch_ok();
+}
+
+int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path) {
+  if (!pool || grid_ctas < 0) return STEP_ERR_INVALID_ARG;
+  if (grid_ctas > 0) pool->attn_grid = grid_ctas;
+  if (fast_path != 0) pool->fast_path = fast_path > 0 ? 1 : -1;
+  return STEP_OK;
+}
+
+}  // extern "C"

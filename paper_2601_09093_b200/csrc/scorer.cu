@@ -1,0 +1,192 @@
+// score_steps: the step scorer at step boundaries and the running-mean trace score.
+//
+//   y = sigmoid(w2 . ReLU(W1 h + b1) + b2)        (Sec. 3.1, "Model Architecture")
+//   score_t = (1/n) sum_{i<=n} y_i^t               (Sec. 3.3)
+//
+// Only rows whose boundary flag is set are scored (Algorithm 1 runs the scorer when the new
+// token ends a step), so the launch is three kernels:
+//   compact : ascending list of boundary rows (block-wide prefix sum), NaN into the other rows
+//   mlp     : for a tile of listed rows and a slice of the m hidden units, the partial
+//             w2 . ReLU(W1 h + b1); hidden rows staged in shared memory as fp32, W1 rows streamed
+//             with 16-byte loads, fp32 accumulation, no rounding of the activations
+//   finish  : fixed-order sum of the slices, + b2, sigmoid, scatter to the row, then the
+//             per-trace (sum, count) update in ascending row order and the refreshed means.
+#include "step_internal.cuh"
+
+#include <math.h>
+
+using namespace stepk;
+
+namespace {
+
+constexpr int kCompactThreads = 1024;
+constexpr int kRowTile = 8;       // listed rows per CTA
+constexpr int kSplits = kScoreSplits;   // slices of the m hidden units
+constexpr int kMlpWarps = 4;
+
+template <typename T> __device__ inline float cvt(T x);
+template <> __device__ inline float cvt<float>(float x) { return x; }
+template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+__global__ void __launch_bounds__(kCompactThreads)
+score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float* __restrict__ step_scores) {
+  __shared__ int s_warp[33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int running = 0;
+  for (int base = 0; base < M; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int f = i < M ? (mask[i] != 0) : 0;
+    int incl = f;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += x;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int w = s_warp[lane];
+      int wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += x;
+      }
+      s_warp[lane] = wi - w;
+      if (lane == 31) s_warp[32] = wi;
+    }
+    __syncthreads();
+    if (f) v.score_idx[running + s_warp[warp] + incl - 1] = i;
+    else if (i < M) step_scores[i] = __int_as_float(0x7fc00000);
+    running += s_warp[32];
+  }
+  if (threadIdx.x == 0) v.counters[C_SCORE_NB] = running;
+}
+
+// grid (kSplits, row tiles).  Dynamic shared memory: kRowTile * D floats.
+template <typename T>
+__global__ void __launch_bounds__(kMlpWarps * 32)
+score_mlp_kernel(DevViews v, const T* __restrict__ hidden, const T* __restrict__ W1, const T* __restrict__ b1,
+                 const T* __restrict__ w2, int D, int m) {
+  extern __shared__ float s_h[];                      // [kRowTile][D]
+  __shared__ float s_part[kMlpWarps][kRowTile];
+  const int nb = v.counters[C_SCORE_NB];
+  const int r0 = blockIdx.y * kRowTile;
+  if (r0 >= nb) return;
+  const int rows = min(kRowTile, nb - r0);
+  const int split = blockIdx.x;
+  const int per = (m + kSplits - 1) / kSplits;
+  const int j0 = split * per, j1 = min(m, j0 + per);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = 0; r < kRowTile; ++r) {
+    if (r < rows) {
+      const T* src = hidden + (size_t)v.score_idx[r0 + r] * D;
+      for (int k = threadIdx.x; k < D; k += blockDim.x) s_h[r * D + k] = cvt(src[k]);
+    } else {
+      for (int k = threadIdx.x; k < D; k += blockDim.x) s_h[r * D + k] = 0.f;
+    }
+  }
+  __syncthreads();
+  float zpart[kRowTile];
+#pragma unroll
+  for (int r = 0; r < kRowTile; ++r) zpart[r] = 0.f;
+  for (int j = j0 + warp; j < j1; j += kMlpWarps) {
+    const T* wrow = W1 + (size_t)j * D;
+    float acc[kRowTile];
+#pragma unroll
+    for (int r = 0; r < kRowTile; ++r) acc[r] = 0.f;
+    for (int k = lane; k < D; k += 32) {
+      const float w = cvt(wrow[k]);
+#pragma unroll
+      for (int r = 0; r < kRowTile; ++r) acc[r] += w * s_h[r * D + k];
+    }
+    const float bj = cvt(b1[j]), wj = cvt(w2[j]);
+#pragma unroll
+    for (int r = 0; r < kRowTile; ++r) {
+      float a = acc[r];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      a += bj;
+      zpart[r] += wj * fmaxf(a, 0.f);
+    }
+  }
+  if (lane == 0)
+    for (int r = 0; r < kRowTile; ++r) s_part[warp][r] = zpart[r];
+  __syncthreads();
+  if (threadIdx.x < rows) {
+    float z = 0.f;
+    for (int w = 0; w < kMlpWarps; ++w) z += s_part[w][threadIdx.x];
+    v.score_z[(size_t)(r0 + threadIdx.x) * kSplits + split] = z;
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
+                    float unscored, float* __restrict__ step_scores) {
+  const int nb = v.counters[C_SCORE_NB];
+  for (int r = threadIdx.x; r < nb; r += blockDim.x) {
+    float z = 0.f;
+    for (int s = 0; s < kSplits; ++s) z += v.score_z[(size_t)r * kSplits + s];
+    z += b2;
+    const float y = 1.f / (1.f + expf(-z));
+    step_scores[v.score_idx[r]] = y;
+    v.score_z[(size_t)r * kSplits] = y;
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
+    float sum = v.score_sum[t];
+    int cnt = v.score_cnt[t];
+    for (int r = 0; r < nb; ++r) {
+      const int row = v.score_idx[r];
+      const int tr = row_trace ? row_trace[row] : row + row_base;
+      if (tr == t) { sum += v.score_z[(size_t)r * kSplits]; ++cnt; }
+    }
+    v.score_sum[t] = sum; v.score_cnt[t] = cnt;
+    v.trace_scores[t] = cnt > 0 ? sum / (float)cnt : unscored;
+  }
+  // rows that name no trace of this pool
+  for (int r = threadIdx.x; r < nb; r += blockDim.x) {
+    const int row = v.score_idx[r];
+    const int tr = row_trace ? row_trace[row] : row + row_base;
+    if (tr < 0 || tr >= g.max_traces) flag_error(v.counters, STEP_ERR_BAD_TRACE);
+  }
+}
+
+}  // namespace
+
+extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* boundary_mask,
+                           const int32_t* row_trace, int M, const scorer_weights* w,
+                           float* step_scores_out, void* stream) {
+  if (!pool || M < 0 || !w) return STEP_ERR_INVALID_ARG;
+  if (M == 0) return STEP_OK;
+  if (!hidden || !boundary_mask || !step_scores_out) return STEP_ERR_INVALID_ARG;
+  if (!w->W1 || !w->b1 || !w->w2 || w->D < 1 || w->m < 1) return STEP_ERR_INVALID_ARG;
+  if (w->dtype != STEP_BF16 && w->dtype != STEP_FP32) return STEP_ERR_INVALID_ARG;
+  const size_t smem = (size_t)kRowTile * w->D * sizeof(float);
+  if (smem > 200 * 1024) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  Geo g = geo_of(pool);
+  const size_t eb = w->dtype == STEP_BF16 ? 2 : 4;
+  for (int off = 0; off < M; off += pool->max_score_rows) {
+    const int Mc = M - off < pool->max_score_rows ? M - off : pool->max_score_rows;
+    const char* hid = (const char*)hidden + (size_t)off * w->D * eb;
+    const int32_t* rt = row_trace ? row_trace + off : nullptr;
+    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, boundary_mask + off, Mc, step_scores_out + off);
+    dim3 grid(kSplits, (Mc + kRowTile - 1) / kRowTile);
+    if (w->dtype == STEP_BF16) {
+      auto kern = score_mlp_kernel<__nv_bfloat16>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+      kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const __nv_bfloat16*)hid, (const __nv_bfloat16*)w->W1,
+                                             (const __nv_bfloat16*)w->b1, (const __nv_bfloat16*)w->w2, w->D, w->m);
+    } else {
+      auto kern = score_mlp_kernel<float>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+      kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const float*)hid, (const float*)w->W1, (const float*)w->b1,
+                                             (const float*)w->w2, w->D, w->m);
+    }
+    // row_trace == NULL means row i is trace i, counted from the start of the whole call
+    score_finish_kernel<<<1, 1024, 0, s>>>(pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off);
+  }
+  return launch_ok();
+}

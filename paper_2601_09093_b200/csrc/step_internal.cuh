@@ -1,0 +1,102 @@
+// Internal definitions shared by the translation units of libstep (never installed).
+//
+// Physical KV layout (private to the library):
+//   kv[layer][block][kv_head][K|V][slot][dim]          slot in [0, page_size)
+// so that one page of one KV head (K rows then V rows) is a single contiguous run of
+// 2 * page_size * head_dim elements - 8 KiB for bf16, page 16, d 128 - which one bulk async
+// copy brings into shared memory.  For bf16 pools whose head_dim is a multiple of 64 the 16-byte
+// chunks of every row are stored XOR-swizzled with the slot number (chunk' = chunk ^ (slot & 7)
+// on the low three bits): the page then lands in shared memory already in the bank-conflict-free
+// arrangement that ldmatrix wants, without a tensor map.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/step.h"
+
+namespace stepk {
+
+constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream partitions of one launch
+constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
+constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
+
+enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4, C_NUM = 64 };
+
+struct MetaLayout {
+  size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;
+  size_t refcount, free_list, claim, counters;
+  size_t append_base, prune_rank, prune_list, prune_off;
+  size_t score_idx, score_z;
+  size_t attn_ml, attn_o;
+  size_t total;
+};
+
+struct DevViews {
+  int32_t* block_table; int32_t* seq_lens; uint8_t* live;
+  float* score_sum; int32_t* score_cnt; float* trace_scores;
+  int32_t* refcount; int32_t* free_list; int32_t* claim; int32_t* counters;
+  int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
+  int32_t* score_idx; float* score_z;
+  float* attn_ml; float* attn_o;
+};
+
+}  // namespace stepk
+
+struct step_pool {
+  kv_pool_config cfg;
+  int G;
+  int elem_bytes;
+  int swizzle;        // 1: rows stored with XOR-swizzled 16-byte chunks
+  int max_score_rows;
+  int next_trace;     // host-side id allocator for forks
+  int num_sms;
+  int attn_grid;      // CTAs of the tensor-core attention launch
+  int fast_path;      // 1 allowed, -1 forced off
+  int device;
+  stepk::MetaLayout lay;
+  stepk::DevViews v;
+};
+
+namespace stepk {
+
+// Geometry handed to kernels by value.
+struct Geo {
+  int L, Hq, Hkv, d, P, num_blocks, max_traces, max_pages, G, swizzle;
+};
+
+inline Geo geo_of(const step_pool* p) {
+  Geo g;
+  g.L = p->cfg.num_layers; g.Hq = p->cfg.num_q_heads; g.Hkv = p->cfg.num_kv_heads;
+  g.d = p->cfg.head_dim; g.P = p->cfg.page_size; g.num_blocks = p->cfg.num_blocks;
+  g.max_traces = p->cfg.max_traces; g.max_pages = p->cfg.max_pages_per_trace;
+  g.G = p->G; g.swizzle = p->swizzle;
+  return g;
+}
+
+// Element offset of (layer, block, head, kv, slot, dim) in kv_storage.
+__host__ __device__ inline size_t kv_page_base(const Geo& g, int layer, int block, int head, int kv) {
+  return ((((size_t)layer * g.num_blocks + block) * g.Hkv + head) * 2 + kv) * ((size_t)g.P * g.d);
+}
+// Offset inside a page of (slot, dim); `cpe` = elements per 16-byte chunk.
+__host__ __device__ inline int kv_in_page(const Geo& g, int slot, int dim, int cpe) {
+  int chunk = dim / cpe, within = dim % cpe;
+  if (g.swizzle) chunk = (chunk & ~7) | ((chunk ^ slot) & 7);
+  return slot * g.d + chunk * cpe + within;
+}
+
+__device__ inline void flag_error(int32_t* counters, int code) {
+  atomicOr(reinterpret_cast<unsigned*>(counters + C_STATUS), 1u << code);
+}
+
+#define STEP_CUDA_OK(expr)                                  \
+  do {                                                      \
+    cudaError_t e__ = (expr);                               \
+    if (e__ != cudaSuccess) return STEP_ERR_CUDA;           \
+  } while (0)
+
+inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? STEP_OK : STEP_ERR_CUDA; }
+
+}  // namespace stepk

@@ -1,0 +1,267 @@
+"""GPU parity: every call of the C ABI against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as OA
+from oracle import scorer as OS
+from paper_2601_09093_b200 import binding as B
+from paper_2601_09093_b200 import harness as H
+from paper_2601_09093_b200 import workloads as W
+
+from gpu_common import Twin, exact_f32, attention_errors
+
+pytestmark = pytest.mark.gpu
+
+# tolerances stated by the benchmark spec for bf16-in / fp32-accumulate attention and for scores
+ATT_MAX, ATT_MEAN, SCORE_TOL = 1e-2, 1e-3, 1e-3
+
+
+def _oracle_attention(tw: Twin, layer, q_exact, n):
+    o = tw.ora
+    return OA.paged_decode_attention(q_exact, o.k_pages[layer], o.v_pages[layer], o.block_table[:n], o.seq_lens[:n])
+
+
+def _gpu_attention(tw: Twin, layer, q_dev, n):
+    v = tw.gpu.views()
+    return tw.gpu.decode_attention(layer, q_dev, v["block_table"][:n], v["seq_lens"][:n])
+
+
+def _build(cfg, suffix, num_blocks=None, shuffle=False, extra_pages=2):
+    P = cfg.page_size
+    n = len(suffix)
+    pages = int(sum(-(-(cfg.prefix_len + s) // P) for s in suffix)) + 8
+    tw = Twin(cfg, num_blocks or pages, max(-(-(cfg.prefix_len + int(max(suffix))) // P) + extra_pages, 4), n, shuffle=shuffle)
+    ids, oids = tw.fork(n, cfg.prefix_len)
+    assert ids == oids
+    for sel, inc in H.ragged_append_plan(np.asarray(suffix)):
+        assert all(tw.append([ids[i] for i in sel], inc))
+    return tw, ids
+
+
+def _check_attention(tw, cfg, n, layers=(0,), max_tol=ATT_MAX, mean_tol=ATT_MEAN):
+    for layer in layers:
+        qb, qx = W.normal(cfg.seed, W.TID_Q, (n, cfg.num_q_heads, cfg.head_dim), cfg.dtype, sub=layer)
+        got = exact_f32(_gpu_attention(tw, layer, H.to_device(qb, cfg.dtype), n))
+        want = _oracle_attention(tw, layer, qx, n)
+        mx, mean = attention_errors(got, want)
+        assert mx <= max_tol and mean <= mean_tol, (layer, mx, mean)
+    assert tw.status() == (0, 0)
+
+
+# ------------------------------------------------------------------ pool
+def test_c0_pool_metadata_and_payload_roundtrip():
+    cfg = W.C0
+    suffix = W.suffix_lengths(cfg)
+    tw, ids = _build(cfg, suffix, num_blocks=cfg.num_blocks)
+    tw.assert_meta_equal()
+    v = tw.gpu.views()
+    for t in (0, 3, 7):
+        S = int(tw.ora.seq_lens[t])
+        k, vv = tw.gpu.read_kv(0, 0, v["block_table"][t], S)
+        K, V = OA.gather_trace_kv(tw.ora.k_pages[0], tw.ora.v_pages[0], tw.ora.block_table[t], S)
+        np.testing.assert_array_equal(exact_f32(k), K[:, 0])
+        np.testing.assert_array_equal(exact_f32(vv), V[:, 0])
+    assert tw.status() == (0, 0)
+
+
+def test_fork_with_partial_page_and_token_by_token_append():
+    cfg = W.scaled(W.C0, prefix_len=37, num_layers=2, num_kv_heads=2, num_q_heads=4)
+    tw = Twin(cfg, 64, 12, 3)
+    ids, oids = tw.fork(3, 37)
+    assert ids == oids == [0, 1, 2]
+    tw.assert_meta_equal()
+    for step in range(30):
+        tw.append(ids, 1)
+    tw.append(ids[:2], 21)
+    tw.assert_meta_equal()
+    _check_attention(tw, cfg, 3, layers=(0, 1), max_tol=1e-4, mean_tol=1e-5)
+
+
+def test_bf16_swizzled_layout_roundtrip_multi_layer():
+    cfg = W.scaled(W.C1, n_traces=3, num_layers=3, prefix_len=40)
+    tw, ids = _build(cfg, [5, 70, 33])
+    tw.assert_meta_equal()
+    v = tw.gpu.views()
+    for layer in range(3):
+        for head in (0, 5, 7):
+            for t in range(3):
+                S = int(tw.ora.seq_lens[t])
+                k, vv = tw.gpu.read_kv(layer, head, v["block_table"][t], S)
+                K, V = OA.gather_trace_kv(tw.ora.k_pages[layer], tw.ora.v_pages[layer], tw.ora.block_table[t], S)
+                np.testing.assert_array_equal(exact_f32(k), K[:, head])
+                np.testing.assert_array_equal(exact_f32(vv), V[:, head])
+
+
+def test_error_conditions_are_flagged_not_fatal():
+    cfg = W.scaled(W.C0, prefix_len=16)
+    tw = Twin(cfg, 3, 2, 3, store_payload=False)
+    ids, _ = tw.fork(2, 16)
+    assert tw.append([0, 1, 5], 16) == [True, True, False]
+    assert tw.status() == (1 << 3, 1 << 3)
+    assert tw.append([0], 1) == [False]
+    assert tw.status() == (1 << 4, 1 << 4)
+    tw.assert_meta_equal()
+    tw2 = Twin(cfg, 2, 4, 2, store_payload=False)
+    tw2.fork(2, 16)
+    assert tw2.append([0, 1], 16) == [True, False]
+    assert tw2.status() == (1 << 2, 1 << 2)
+    tw2.assert_meta_equal()
+    # a fork the free list cannot serve is a no-op
+    tw3 = Twin(cfg, 1, 4, 2, store_payload=False)
+    tw3.gpu.fork_prefix(2, 32, torch.zeros((1, 1, 32, 64), device="cuda"), torch.zeros((1, 1, 32, 64), device="cuda"))
+    assert tw3.gpu.last_error()[1] == 1 << 2 and tw3.gpu.stats() == dict(used=0, free=1, total=1, live_traces=0)
+
+
+def test_host_side_argument_checks():
+    pool = H.make_pool(W.C0, 8, 4)
+    z = torch.zeros(4, device="cuda")
+    with pytest.raises(B.StepError):
+        pool.prune_if_saturated(None, 0.95, 0.0)
+    with pytest.raises(B.StepError):
+        pool.prune_if_saturated(None, 1.5, 0.5)
+    with pytest.raises(B.StepError):
+        pool.decode_attention(3, z, z, z)
+    with pytest.raises(B.StepError):
+        B.kv_pool_required_bytes(num_layers=1, num_q_heads=3, num_kv_heads=2, head_dim=64, page_size=16,
+                                 num_blocks=4, max_traces=1, max_pages_per_trace=1, dtype=0)
+
+
+# ------------------------------------------------------------------ attention
+def test_c0_attention_fp32():
+    cfg = W.C0
+    tw, ids = _build(cfg, W.suffix_lengths(cfg), num_blocks=cfg.num_blocks)
+    _check_attention(tw, cfg, cfg.n_traces, max_tol=1e-4, mean_tol=1e-5)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (64, 8), (8, 8), (16, 1), (24, 2)])
+def test_bf16_attention_ragged_small(Hq, Hkv):
+    # several pages per warp partition, partial last pages, a one-token and an empty trace
+    cfg = W.scaled(W.C1, n_traces=9, num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=48)
+    suffix = [0, 1, 15, 16, 17, 700, 2049, 333, 5000]
+    tw, ids = _build(cfg, suffix)
+    _check_attention(tw, cfg, 9)
+    # same inputs through the scalar kernel
+    tw.gpu.set_attention_config(fast_path=-1)
+    _check_attention(tw, cfg, 9)
+
+
+def test_bf16_attention_empty_and_single_token_traces():
+    cfg = W.scaled(W.C1, n_traces=4, prefix_len=0)
+    tw = Twin(cfg, 16, 4, 4)
+    ids, _ = tw.fork(4, 0)
+    tw.append([1], 1)
+    tw.append([3], 20)
+    _check_attention(tw, cfg, 4)
+    v = tw.gpu.views()
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (4, 32, 128), "bf16")
+    out = exact_f32(_gpu_attention(tw, 0, H.to_device(qb, "bf16"), 4))
+    assert np.all(out[0] == 0) and np.all(out[2] == 0)
+    k, vv = tw.gpu.read_kv(0, 2, v["block_table"][1], 1)
+    np.testing.assert_allclose(out[1, 8:12], np.tile(exact_f32(vv), (4, 1)), atol=1e-6)   # S = 1: o = V[0]
+
+
+def test_attention_grid_sizes_and_page_shuffle_agree():
+    # page-permutation invariance on the GPU, and independence from how the KV stream is partitioned
+    cfg = W.scaled(W.C1, n_traces=6, prefix_len=64)
+    suffix = [100, 900, 2500, 31, 1200, 64]
+    outs = []
+    for shuffle in (False, True):
+        tw, ids = _build(cfg, suffix, num_blocks=512, shuffle=shuffle)
+        qb, qx = W.normal(cfg.seed, W.TID_Q, (6, 32, 128), "bf16")
+        qd = H.to_device(qb, "bf16")
+        want = _oracle_attention(tw, 0, qx, 6)
+        for grid in (0, 1, 3, 37, 500):
+            tw.gpu.set_attention_config(grid_ctas=grid)
+            got = exact_f32(_gpu_attention(tw, 0, qd, 6))
+            mx, mean = attention_errors(got, want)
+            assert mx <= ATT_MAX and mean <= ATT_MEAN, (shuffle, grid, mx, mean)
+            outs.append(got)
+        assert tw.status() == (0, 0)
+    assert np.abs(outs[0] - outs[5]).max() < 1e-5      # only the physical placement differs
+
+
+def test_attention_padding_slots_do_not_leak():
+    # unused slots of the last page hold NaN bit patterns: the result must not see them
+    cfg = W.scaled(W.C1, n_traces=2, prefix_len=0)
+    tw = Twin(cfg, 8, 4, 2)
+    tw.gpu.kv_storage.view(torch.int16).fill_(0x7FC0)   # bf16 NaN everywhere
+    tw.fork(2, 0)
+    tw.append([0, 1], 5)
+    tw.append([1], 13)
+    _check_attention(tw, cfg, 2)
+
+
+def test_bad_block_table_is_flagged():
+    cfg = W.scaled(W.C1, n_traces=1, prefix_len=32)
+    tw, ids = _build(cfg, [40])
+    v = tw.gpu.views()
+    bt = v["block_table"][:1].clone()
+    bt[0, 1] = 10 ** 6
+    q = torch.zeros((1, 32, 128), dtype=torch.bfloat16, device="cuda")
+    tw.gpu.decode_attention(0, q, bt, v["seq_lens"][:1])
+    assert tw.gpu.last_error()[1] == 1 << 7
+
+
+# ------------------------------------------------------------------ scorer
+def _scorer_case(cfg, M, density, row_trace=None, bias=0.05, max_traces=None, max_score_rows=0):
+    T = max_traces or cfg.n_traces
+    pool = H.make_pool(cfg, 8, 4, T, max_score_rows=max_score_rows)
+    (W1b, W1x), (b1b, b1x), (w2b, w2x), b2 = W.scorer_weights(cfg, bias_std=bias)
+    wts = B.ScorerWeights(H.to_device(W1b, cfg.dtype), H.to_device(b1b, cfg.dtype), H.to_device(w2b, cfg.dtype), b2,
+                          H.step_dtype(cfg))
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (M, cfg.scorer_D), cfg.dtype)
+    mask = W.boundary_mask(cfg, M, density=density)
+    rt_dev = None if row_trace is None else torch.from_numpy(row_trace.astype(np.int32)).cuda()
+    got = pool.score_steps(H.to_device(hb, cfg.dtype), torch.from_numpy(mask).cuda(), rt_dev, wts)
+    want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+    g = got.cpu().numpy()
+    assert np.isnan(g[mask == 0]).all()
+    if mask.any():
+        assert np.abs(g[mask == 1] - want[mask == 1]).max() <= SCORE_TOL
+    ts = OS.TraceScores(T)
+    ts.update(g, mask, row_trace)                       # running means from the GPU's own step scores
+    v = pool.views()
+    np.testing.assert_allclose(v["trace_scores"].cpu().numpy(), ts.scores(), atol=1e-6)
+    np.testing.assert_array_equal(v["score_cnt"].cpu().numpy(), ts.cnt)
+    ts2 = OS.TraceScores(T)
+    ts2.update(want, mask, row_trace)                   # and within tolerance of the all-oracle means
+    assert np.abs(v["trace_scores"].cpu().numpy() - ts2.scores()).max() <= SCORE_TOL
+    assert pool.last_error() == (0, 0)
+    return pool, wts, g, mask
+
+
+def test_c0_scorer_fp32():
+    _scorer_case(W.C0, 8, 1.0, bias=0.0)
+
+
+def test_scorer_bf16_decode_shape():
+    _scorer_case(W.C1, 64, 1.0 / 8)
+
+
+def test_scorer_bf16_all_and_none_boundaries():
+    _scorer_case(W.C1, 64, 1.0)
+    _scorer_case(W.C1, 64, 0.0)
+
+
+def test_scorer_batched_rows_with_row_trace_and_chunking():
+    cfg = W.C1
+    M = 64 * 40 + 13
+    rt = (np.arange(M) % 64).astype(np.int32)
+    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M)
+    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=1000)    # several launches
+
+
+def test_scorer_c4_shape():
+    _scorer_case(W.C4, 128, 0.1)
+
+
+def test_scorer_running_mean_accumulates_across_calls():
+    cfg = W.C1
+    pool, wts, g1, m1 = _scorer_case(cfg, 64, 0.5)
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (64, cfg.scorer_D), cfg.dtype, sub=7)
+    mask = W.boundary_mask(cfg, 64, sub=7, density=0.5)
+    g2 = pool.score_steps(H.to_device(hb, cfg.dtype), torch.from_numpy(mask).cuda(), None, wts).cpu().numpy()
+    ts = OS.TraceScores(64)
+    ts.update(g1, m1); ts.update(g2, mask)
+    np.testing.assert_allclose(pool.views()["trace_scores"].cpu().numpy(), ts.scores(), atol=1e-6)
