@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the STEP decode hot path (libstep) on B200.
+
+A "step" is one decode iteration of Algorithm 1 for all live traces on device-resident state:
+append_kv (one new token per trace, all layers) -> decode_attention for every layer ->
+score_steps on the step-end hidden states -> prune_if_saturated.
+
+Default workload: the 64-trace memory-saturated configuration (Qwen3-8B KV layout, 36 layers,
+8 KV heads, d = 128, bf16, page 16, pool of ~150 GB) in the state just below the 95 % trigger,
+i.e. the headline state of the prune benchmark.  Inputs are synthetic and seeded.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "paged decode-attn KV GB/s (fraction of B200 HBM peak); trace-decode-steps/sec"
+UNIT = "trace-decode-steps/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4"])
+    ap.add_argument("--num-blocks", type=int, default=0, help="override the pool size (blocks)")
+    ap.add_argument("--grid", type=int, default=0, help="CTAs of the attention launch (0 = library default)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thr = threading.Thread(target=self._read, daemon=True)
+            self.thr.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+def workload_plan(name, num_blocks_override, steps_total, free_bytes=None):
+    """Shapes of the benchmark state: config, per-trace suffix lengths, pool size."""
+    from paper_2601_09093_b200 import workloads as W
+    if name == "c3":
+        cfg = W.C3
+        nb = num_blocks_override or cfg.num_blocks
+        block_bytes = cfg.bytes_per_token * cfg.page_size
+        if free_bytes is not None:
+            fit = int((free_bytes - (6 << 30)) // block_bytes)
+            nb = min(nb, fit)
+        limit = math.floor(float(np.float32(cfg.threshold)) * nb)
+        shared = cfg.prefix_len // cfg.page_size
+        margin_pages = -(-steps_total // cfg.page_size) + 1
+        p0 = (limit - shared) // cfg.n_traces - margin_pages         # private pages per trace at the start
+        if p0 < 1:
+            raise SystemExit("pool too small for the memory-saturated workload")
+        suffix = np.full(cfg.n_traces, p0 * cfg.page_size, dtype=np.int64)
+        max_pages = shared + p0 + margin_pages + 2
+        return cfg, suffix, nb, max_pages, cfg.num_layers
+    cfg = {"c1": W.C1, "c2": W.C2, "c4": W.C4}[name]
+    suffix = W.suffix_lengths(cfg)
+    pages = int(sum(-(-(cfg.prefix_len + s + steps_total) // cfg.page_size) for s in suffix)) + 64
+    nb = num_blocks_override or pages
+    max_pages = -(-(cfg.prefix_len + int(suffix.max()) + steps_total) // cfg.page_size) + 2
+    phys_layers = cfg.num_layers
+    if free_bytes is not None:
+        per_layer = nb * cfg.bytes_per_token_layer * cfg.page_size
+        phys_layers = max(1, min(cfg.num_layers, int((free_bytes - (6 << 30)) // per_layer)))
+    return cfg, suffix, nb, max_pages, phys_layers
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_09093_b200 import binding as B, harness as H, workloads as W
+    from paper_2601_09093_b200 import build as _build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        _build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    B.lib()
+
+    K, Wm = args.steps, max(args.warmup, 3)
+    e2e_steps = 0 if args.no_e2e else K
+    steps_total = Wm + K + (Wm + e2e_steps) + 4
+    free_b, total_b = torch.cuda.mem_get_info(dev)
+    cfg, suffix, nb, max_pages, phys_layers = workload_plan(args.workload, args.num_blocks, steps_total, free_b)
+    cfg_pool = W.scaled(cfg, num_layers=phys_layers)
+    T, L = cfg.n_traces, cfg.num_layers
+    pool = H.make_pool(cfg_pool, nb, max_pages, T, max_score_rows=T, device=dev)
+    if args.grid:
+        pool.set_attention_config(grid_ctas=args.grid)
+    if cfg.shuffle_pages:
+        H.shuffle_free_list(pool, cfg.seed + rank)
+    t_fill = time.time()
+    ids = H.fill_random_device(pool, cfg_pool, suffix, seed=cfg.seed + 7919 * rank,
+                               chunk_tokens=max(16, (1 << 28) // (T * cfg_pool.bytes_per_token)))
+    torch.cuda.synchronize()
+    t_fill = time.time() - t_fill
+    v = pool.views()
+    ids_dev = torch.tensor(ids, dtype=torch.int32, device=dev)
+
+    # rotating sets of per-step inputs (device copies and pinned host copies of the same values)
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 1 + rank)
+    NSETS = 2
+    def rnd(*shape):
+        return torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    sets = []
+    mask_np = [W.boundary_mask(cfg, T, sub=100 + i) for i in range(NSETS)]
+    for i in range(NSETS):
+        s = dict(q=rnd(L, T, cfg.num_q_heads, cfg.head_dim), k=rnd(T, 1, phys_layers, cfg.num_kv_heads, cfg.head_dim),
+                 v=rnd(T, 1, phys_layers, cfg.num_kv_heads, cfg.head_dim), h=rnd(T, cfg.scorer_D),
+                 m=torch.from_numpy(mask_np[i]).to(dev))
+        s["host"] = {k: s[k].cpu().pin_memory() for k in ("q", "k", "v", "h", "m")}
+        sets.append(s)
+    (W1b, _), (b1b, _), (w2b, _), b2 = W.scorer_weights(cfg)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16", dev), H.to_device(b1b, "bf16", dev), H.to_device(w2b, "bf16", dev), b2, B.STEP_BF16)
+    out = torch.empty((L, T, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
+    step_scores = torch.empty(T, dtype=torch.float32, device=dev)
+    host_out = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    host_scores = torch.empty(T, dtype=torch.float32).pin_memory()
+    host_tscores = torch.empty(pool.max_traces, dtype=torch.float32).pin_memory()
+    host_npruned = torch.empty(1, dtype=torch.int32).pin_memory()
+    stream = torch.cuda.current_stream()
+    attn_events = []
+
+    def hot_path(s, time_attn=False):
+        pool.append_kv(ids_dev, 1, s["k"], s["v"])
+        for l in range(L):
+            if time_attn:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            pool.decode_attention(l % phys_layers, s["q"][l], v["block_table"], v["seq_lens"], out[l])
+            if time_attn:
+                e1.record(stream); attn_events.append((e0, e1))
+        pool.score_steps(s["h"], s["m"], None, wts, step_scores)
+        pool.prune_if_saturated(None, cfg.threshold, cfg.keep_frac)
+
+    def e2e_step(s, dst):
+        for k in ("q", "k", "v", "h", "m"):
+            dst[k].copy_(s["host"][k], non_blocking=True)
+        hot_path(dst)
+        host_out.copy_(out, non_blocking=True)
+        host_scores.copy_(step_scores, non_blocking=True)
+        host_tscores.copy_(v["trace_scores"], non_blocking=True)
+        host_npruned.copy_(pool.n_pruned, non_blocking=True)
+        stream.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(Wm):
+        hot_path(sets[i % NSETS])
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for i in range(K):
+        hot_path(sets[i % NSETS], time_attn=True)
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev0.elapsed_time(ev1)
+    attn_ms = [a.elapsed_time(b) for a, b in attn_events]
+    err_code, err_mask = pool.last_error()
+    n_live = pool.stats()["live_traces"]
+    seq_now = v["seq_lens"][:T].cpu().numpy().astype(np.int64)
+
+    # ---- end to end: host buffers in, host results out, every step
+    e2e = None
+    if e2e_steps:
+        dst = {k: torch.empty_like(sets[0][k]) for k in ("q", "k", "v", "h", "m")}
+        for i in range(Wm):
+            e2e_step(sets[i % NSETS], dst)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(sets[i % NSETS], dst)
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        h2d = sum(sets[0]["host"][k].numel() * sets[0]["host"][k].element_size() for k in ("q", "k", "v", "h", "m"))
+        d2h = host_out.numel() * 4 + host_scores.numel() * 4 + host_tscores.numel() * 4 + 4
+        e2e = (e2e_s, h2d, d2h)
+
+    if world > 1:
+        tt = torch.tensor([ms_total, e2e[0] if e2e else 0.0], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt[0]); e2e = (float(tt[1]), e2e[1], e2e[2]) if e2e else None
+        ok = torch.tensor([int(err_mask == 0 and n_live == T)], device=dev)
+        dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+        all_ok = bool(ok.item())
+    else:
+        all_ok = err_mask == 0 and n_live == T
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (decode_attention of one layer)
+    peak, peak_kind = measured_peaks()
+    mid_suffix = seq_now - cfg.prefix_len - K // 2          # lengths at the middle of the timed region
+    kv_bytes = H.unique_kv_bytes(cfg, cfg.prefix_len, mid_suffix)
+    pages = int(np.sum(-(-(mid_suffix + cfg.prefix_len) // cfg.page_size)))
+    algo_bytes = kv_bytes + T * cfg.num_q_heads * cfg.head_dim * (2 + 4) + pages * 4
+    attn_avg_ms = float(np.mean(attn_ms))
+    achieved = algo_bytes / (attn_avg_ms * 1e-3) / 1e9
+    value = world * T * K / (ms_total * 1e-3)
+    res = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic (seeded, drawn on device)",
+        "config": {"workload": cfg.name, "traces": T, "layers": L, "layers_resident": phys_layers,
+                   "q_heads": cfg.num_q_heads, "kv_heads": cfg.num_kv_heads, "head_dim": cfg.head_dim,
+                   "page": cfg.page_size, "num_blocks": nb, "pool_gb": round(pool.kv_bytes / 1e9, 2),
+                   "tokens_per_trace": int(np.mean(seq_now)), "threshold": cfg.threshold, "keep_frac": cfg.keep_frac,
+                   "l2_policy": "inputs larger than L2 (%.1f GB of KV per layer call)" % (kv_bytes / 1e9),
+                   "multi_gpu": "replicas only (one independent problem per GPU)", "fill_s": round(t_fill, 1)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                     "kernel": "decode_attention (attn_mma_kernel + attn_merge_kernel), one layer",
+                     "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": attn_avg_ms,
+                     "min_launch_ms": float(np.min(attn_ms)), "launches_timed": len(attn_ms)},
+        "kv_gbs": achieved, "attention_share_of_step": float(np.sum(attn_ms)) / ms_total,
+        "gpu_launches": K * (2 + 2 * L + 3 + 1), "clocks": clocks,
+        "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
+    }
+    if e2e:
+        res["e2e"] = {"value": world * T * e2e_steps / e2e[0], "unit": UNIT, "h2d_bytes_per_step": e2e[1],
+                      "d2h_bytes_per_step": e2e[2], "ms_per_step": e2e[0] * 1e3 / e2e_steps}
+    if not args.no_cpu_baseline:
+        res["cpu_baseline"], res["sampled_parity"] = cpu_baseline_and_parity(pool, cfg, sets[(K - 1) % NSETS], out, L, phys_layers)
+    print(json.dumps(res))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0):
+    """Times the oracle on a bounded sample of the benchmark's own state and checks the GPU against it.
+
+    Sample: whole (trace, layer) attentions - all KV heads and query heads of a trace in one layer -
+    taken round-robin over layers {last, first, middle, ...} and over all traces until about
+    `cpu_budget_s` seconds of oracle time are spent.  The stored K/V rows are read back through
+    kv_pool_read_kv so that the oracle sees the very bytes the kernel read.  CPU throughput is
+    extrapolated to whole trace-decode-steps by the layer count.
+    """
+    import torch
+    from oracle import attention as OA
+    v = pool.views()
+    T = cfg.n_traces
+    layers = [L - 1, 0, L // 2] + [l for l in range(1, L - 1) if l != L // 2]
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    t_cpu, max_err, sum_err, cnt, done = 0.0, 0.0, 0.0, 0, 0
+    wall0 = time.perf_counter()
+    for layer in layers[:L]:
+        # the output of this layer for the inputs in `s`, recomputed so that it is known to match them
+        pool.decode_attention(layer % phys_layers, s["q"][layer], v["block_table"], v["seq_lens"], out[layer])
+        torch.cuda.synchronize()
+        got_all = out[layer].cpu().numpy().astype(np.float64)
+        q_all = s["q"][layer].float().cpu().numpy().astype(np.float64)
+        for t in range(T):
+            S = int(v["seq_lens"][t].item())
+            K_ = np.empty((S, cfg.num_kv_heads, cfg.head_dim), dtype=np.float64)
+            V_ = np.empty_like(K_)
+            for h in range(cfg.num_kv_heads):
+                k, vv = pool.read_kv(layer % phys_layers, h, v["block_table"][t], S)
+                K_[:, h] = k.float().cpu().numpy(); V_[:, h] = vv.float().cpu().numpy()
+            t0 = time.perf_counter()
+            want = OA.dense_decode_attention(q_all[t], K_, V_)
+            t_cpu += time.perf_counter() - t0
+            err = np.abs(got_all[t] - want)
+            max_err = max(max_err, float(err.max())); sum_err += float(err.sum()); cnt += err.size
+            done += 1
+            if t_cpu >= cpu_budget_s or time.perf_counter() - wall0 > 90.0:
+                break
+        if t_cpu >= cpu_budget_s or time.perf_counter() - wall0 > 90.0:
+            break
+    value = done / (t_cpu * L)
+    base = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d (trace, layer) attentions at full length, all heads (%.1f s of CPU), extrapolated to %d layers per step"
+                      % (done, t_cpu, L)}
+    par = {"what": "decode_attention vs fp64 oracle on read-back KV: %d (trace, layer) pairs, all heads" % done,
+           "max_abs_err": max_err, "mean_abs_err": sum_err / cnt, "tolerance": {"max": 1e-2, "mean": 1e-3},
+           "ok": bool(max_err <= 1e-2 and sum_err / cnt <= 1e-3)}
+    return base, par
+
+
+# ---------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The reference arm of this build is the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import attention as OA, scorer as OS
+    from oracle.kv_pool import KVPoolOracle
+    from paper_2601_09093_b200 import workloads as W
+
+    K, Wm = args.steps, max(args.warmup, 1)
+    cfg, suffix, nb, max_pages, _ = workload_plan(args.workload, args.num_blocks, Wm + K + 4)
+    T, L, P = cfg.n_traces, cfg.num_layers, cfg.page_size
+    # bounded sample of one step: attention of ONE trace in ONE layer at the benchmark's length,
+    # the scorer on the step's boundary rows, the pool bookkeeping and the trigger for all traces
+    S = cfg.prefix_len + int(suffix[0])
+    pool = KVPoolOracle(L, cfg.num_kv_heads, cfg.head_dim, P, nb, T, max_pages, store_payload=False)
+    ids = pool.fork_prefix(T, cfg.prefix_len)
+    pool.append_kv(ids, int(suffix[0]))
+    kb, Kx = W.normal(cfg.seed, W.TID_K, (S + Wm + K + 4, cfg.num_kv_heads, cfg.head_dim), "bf16")
+    vb, Vx = W.normal(cfg.seed, W.TID_V, (S + Wm + K + 4, cfg.num_kv_heads, cfg.head_dim), "bf16")
+    Kx, Vx = Kx.astype(np.float64), Vx.astype(np.float64)
+    (_, W1x), (_, b1x), (_, w2x), b2 = W.scorer_weights(cfg)
+    ts = OS.TraceScores(T)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+
+    SAMPLE = 8
+
+    def step(i):
+        nonlocal S
+        pool.append_kv([t for t in range(T) if pool.live[t]], 1)
+        S += 1
+        for j in range(SAMPLE):                         # SAMPLE (trace, layer) attentions at full length
+            _, qx = W.normal(cfg.seed, W.TID_Q, (cfg.num_q_heads, cfg.head_dim), "bf16", sub=i * SAMPLE + j)
+            OA.dense_decode_attention(qx, Kx[:S], Vx[:S])
+        _, hx = W.normal(cfg.seed, W.TID_HID, (T, cfg.scorer_D), "bf16", sub=i)
+        mask = W.boundary_mask(cfg, T, sub=100 + i)
+        ys = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+        ts.update(ys, mask)
+        pool.prune_if_saturated(ts.scores().astype(np.float32), cfg.threshold, cfg.keep_frac, on_evict=ts.clear)
+
+    for i in range(Wm):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(K):
+        step(Wm + i)
+    dt = time.perf_counter() - t0
+    # one sample step covers SAMPLE of the T*L trace-layer attentions of a full step
+    value = K * SAMPLE / (dt * L)                                   # whole trace-decode-steps per second
+    res = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+           "warmup": Wm, "ms_per_step": dt * 1e3 / K, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+           "config": {"workload": cfg.name, "traces": T, "layers": L, "tokens_per_trace": S,
+                      "note": "CPU oracle; each step is a bounded sample"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                            "sample": "per step: %d (trace, layer) attentions (all heads) at full length, scorer on the " % SAMPLE +
+                                      ("boundary rows, pool bookkeeping + trigger for all traces; extrapolated by x%d layers" % L)},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
