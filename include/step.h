@@ -120,6 +120,32 @@ int decode_attention(step_pool* pool, int layer, const void* q,
                      const int32_t* block_table, const int32_t* seq_lens, int n,
                      void* out, void* stream);
 
+/* decode_attention without any caller-provided or allocated scratch.  (The paper has no
+ * counterpart: this entry point exists for hosts, not for the method.)
+ *
+ * Same result as decode_attention, for callers that cannot obtain device memory when they need
+ * attention: a plug-in running inside another framework's pool-managed region, a serving loop that
+ * bans allocator calls after start-up, an embedder that can only pass the buffers it was given.
+ * The kernel's split partials live in a fixed array inside the library image (about 9.9 MB per GPU
+ * that loads the library, held until the process exits); the call itself performs no cudaMalloc /
+ * cudaFree and calls no allocating routine.
+ *
+ * Limits (fixed by that array): bf16 pools with head_dim 128 and page_size 16 only (else
+ * STEP_ERR_INVALID_ARG); num_q_heads / num_kv_heads <= 8 and n <= 2048, else STEP_ERR_CAPACITY with
+ * nothing launched.  The launch uses at most 148 CTAs whatever kv_pool_set_attention_config says.
+ * The pool's device must be the current device.
+ *
+ * First use on a device: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) before it launches.  Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device - from every pool and every stream - use the same array, and it
+ * keeps whatever the previous call left.  Nothing in it has to start at zero (each call writes every
+ * partial before it reads it), but two calls that overlap in time on the GPU race on it: keep
+ * calls of this entry point ordered, e.g. on one stream. */
+int decode_attention_static(step_pool* pool, int layer, const void* q,
+                            const int32_t* block_table, const int32_t* seq_lens, int n,
+                            void* out, void* stream);
+
 /* Step scorer at step boundaries (Sec. 3.1) and running-mean update (Sec. 3.3):
  * for every row i with boundary_mask[i] != 0:
  *   y = sigmoid(w2 . ReLU(W1 hidden[i] + b1) + b2);  step_scores_out[i] = y;

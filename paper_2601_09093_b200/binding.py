@@ -62,6 +62,7 @@ def lib():
     L.kv_pool_fork_prefix.argtypes = [vp, i, i, vp, vp, ip, vp]
     L.append_kv.argtypes = [vp, vp, i, i, vp, vp, vp]
     L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.decode_attention_static.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
     L.prune_if_saturated.argtypes = [vp, vp, C.c_float, C.c_float, vp, vp, vp]
     L.kv_pool_release_traces.argtypes = [vp, vp, i, vp]
@@ -179,6 +180,12 @@ class KVPool:
             out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
         _check("decode_attention", lib().decode_attention(self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens),
                                                           n, _ptr(out), _stream(stream)))
+        return out
+
+    def decode_attention_static(self, layer, q, block_table, seq_lens, out, stream=None):
+        """The allocation-free variant: `out` must be supplied by the caller; nothing is allocated."""
+        _check("decode_attention_static", lib().decode_attention_static(self.handle, layer, _ptr(q), _ptr(block_table),
+                                                                        _ptr(seq_lens), q.shape[0], _ptr(out), _stream(stream)))
         return out
 
     def score_steps(self, hidden, boundary_mask, row_trace, weights, step_scores_out=None, stream=None):

@@ -583,3 +583,83 @@ extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const
         pool->v.counters);
   return launch_ok();
 }
+
+// =============================================================== allocation-free variant
+// decode_attention_static: the tensor-core kernel above with its (m, l, o) partials kept in a
+// fixed array that is part of the library image instead of in caller-provided metadata.
+//
+// Who needs it: code that must run attention but is not allowed to obtain device memory at that
+// point - e.g. a plug-in called inside someone else's memory-pool-managed region, a real-time loop
+// that forbids allocator calls after start-up, or a host that hands this library buffers it cannot
+// grow.  Such a caller passes only inputs and the output; nothing here calls cudaMalloc, cudaFree
+// or any allocating routine.
+//
+// The scratch is a file-scope __device__ array of a fixed, modest size (kStaticScratchFloats
+// floats, about 9.9 MB); every GPU that loads the library carries it until the process exits.
+// In host code the array's NAME is only a stand-in symbol, not a device address, so the launcher
+// asks the runtime for the real address once per device (cudaGetSymbolAddress, with that device
+// current, return code checked) and passes that pointer to the kernels.
+namespace {
+
+constexpr int kStaticMaxPartitions = 1184;   // 148 SMs x 8 warps
+constexpr int kStaticMaxG = 8;               // query heads per KV head
+constexpr size_t kStaticMlFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * 2;
+constexpr size_t kStaticOFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * kD;
+constexpr size_t kStaticScratchFloats = kStaticMlFloats + kStaticOFloats;
+
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device; null until set up
+
+// Set-up, once per device: resolve the device address of the scratch symbol.
+int static_scratch_for_current_device(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return STEP_ERR_CUDA;
+  float* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess || !p) return STEP_ERR_CUDA;
+    __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);   // same value whoever wins
+  }
+  *out = p;
+  return STEP_OK;
+}
+
+}  // namespace
+
+extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                       const int32_t* seq_lens, int n, void* out, void* stream) {
+  if (!pool || n < 0) return STEP_ERR_INVALID_ARG;
+  if (n == 0) return STEP_OK;
+  if (!q || !block_table || !seq_lens || !out) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  if (layer < 0 || layer >= g.L) return STEP_ERR_INVALID_ARG;
+  // only the shape the tensor-core kernel covers
+  if (pool->cfg.dtype != STEP_BF16 || g.d != kD || g.P != kP || !pool->swizzle) return STEP_ERR_INVALID_ARG;
+  // sizes beyond what the fixed scratch holds
+  if (g.G > kStaticMaxG || n > kMaxTracesFast) return STEP_ERR_CAPACITY;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STEP_ERR_CUDA;
+  if (dev != pool->device) return STEP_ERR_INVALID_ARG;   // the pool's device must be current
+  float* scratch = nullptr;
+  const int st = static_scratch_for_current_device(&scratch);
+  if (st != STEP_OK) return st;
+  int grid = pool->attn_grid;
+  if (grid * kWarpsDefault > kStaticMaxPartitions) grid = kStaticMaxPartitions / kWarpsDefault;
+  if (grid < 1) grid = 1;
+  AttnArgs a;
+  a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
+  a.q = (const __nv_bfloat16*)q;
+  a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
+  a.ws_ml = scratch; a.ws_o = scratch + kStaticMlFloats; a.counters = pool->v.counters;
+  a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
+  const size_t smem = (size_t)kWarpsDefault * kStagesDefault * kPageBytes + (size_t)kWarpsDefault * kStagesDefault * 8 +
+                      (size_t)(n + 1) * 4;
+  auto kern = attn_mma_kernel<kWarpsDefault, kStagesDefault, false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  kern<<<grid, kWarpsDefault * 32, smem, s>>>(a);
+  attn_merge_kernel<<<dim3(a.Hkv, a.n), kD, 0, s>>>(a, grid * kWarpsDefault);
+  return launch_ok();
+}

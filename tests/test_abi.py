@@ -1,0 +1,68 @@
+"""The C-ABI library builds, loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if not fn.endswith(".h"):
+            continue
+        src = open(os.path.join(inc, fn)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names += re.findall(r"^\s*(?:const\s+char\s*\*|int|size_t)\s+(\w+)\s*\(", src, flags=re.M)
+    return names
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2601_09093_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+def test_header_declares_the_hot_path_calls():
+    names = _declared_functions()
+    for required in ("kv_pool_create", "kv_pool_fork_prefix", "append_kv", "decode_attention", "score_steps",
+                     "prune_if_saturated", "kv_pool_required_bytes", "kv_pool_destroy"):
+        assert required in names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), "libstep.so does not export " + n
+
+
+def test_required_bytes_needs_no_gpu():
+    from paper_2601_09093_b200 import binding as B
+    kv, meta = B.kv_pool_required_bytes(num_layers=36, num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16,
+                                        num_blocks=65536, max_traces=64, max_pages_per_trace=16384, dtype=B.STEP_BF16)
+    assert kv == 65536 * 16 * 147456                  # 144 KiB per token, 2.25 MiB per block
+    assert 0 < meta < 64 << 20
+    with pytest.raises(B.StepError):
+        B.kv_pool_required_bytes(num_layers=1, num_q_heads=5, num_kv_heads=2, head_dim=128, page_size=16,
+                                 num_blocks=1, max_traces=1, max_pages_per_trace=1, dtype=B.STEP_BF16)
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2601_09093_b200 import binding as B
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libstep.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        B.lib()
+
+
+def test_product_path_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2601_09093_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src.replace("the oracle", "").replace("CPU oracle", ""), f
