@@ -121,8 +121,10 @@ def workload_plan(name, num_blocks_override, steps_total, free_bytes=None):
         return cfg, suffix, nb, max_pages, cfg.num_layers
     cfg = {"c1": W.C1, "c2": W.C2, "c4": W.C4}[name]
     suffix = W.suffix_lengths(cfg)
-    pages = int(sum(-(-(cfg.prefix_len + s + steps_total) // cfg.page_size) for s in suffix)) + 64
-    nb = num_blocks_override or pages
+    shared = cfg.prefix_len // cfg.page_size
+    pages = shared + int(sum(-(-(s + steps_total) // cfg.page_size) + 1 for s in suffix))
+    # these workloads time attention at a fixed trace set: size the pool so the trigger stays quiet
+    nb = num_blocks_override or int(pages / float(np.float32(cfg.threshold)) * 1.02) + 64
     max_pages = -(-(cfg.prefix_len + int(suffix.max()) + steps_total) // cfg.page_size) + 2
     phys_layers = cfg.num_layers
     if free_bytes is not None:
