@@ -196,6 +196,16 @@ int kv_pool_read_kv(step_pool* pool, int layer, int kv_head, const int32_t* bloc
 /* Tuning knobs of decode_attention (0 keeps the current value): CTAs per launch, and whether
  * the tensor-core bf16 path may be used (1) or the scalar kernel is forced (-1). */
 int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path);
+/* Which first-layer kernel score_steps uses for bf16 scorers whose shape the tensor-core kernel covers
+ * (D a multiple of 64, m a multiple of 64 and <= 1024, 16-byte aligned W1 and hidden): mode 0 (default)
+ * sends a launch to the tensor cores when it has at least tc_min_rows boundary rows (the count is taken
+ * on the device) and to the CUDA-core kernel otherwise; mode 1 always uses the tensor cores, mode -1 never.
+ * tc_min_rows = 0 keeps the current value (default 128). */
+int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows);
+/* What the most recent score_steps launch did (of its last chunk, if M exceeded max_score_rows):
+ * *n_rows = boundary rows it found, *tc_units = hidden units per CTA of the tensor-core kernel, or 0 if
+ * the CUDA-core kernel scored the rows.  Host ints, either may be NULL; synchronises the stream. */
+int kv_pool_score_launch_info(step_pool* pool, int* n_rows, int* tc_units, void* stream);
 /* Library build tag, for logs. */
 const char* step_version(void);
 

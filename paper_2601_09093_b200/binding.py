@@ -72,6 +72,8 @@ def lib():
     L.kv_pool_last_error.argtypes = [vp, C.POINTER(C.c_uint), vp]
     L.kv_pool_read_kv.argtypes = [vp, i, i, vp, i, vp, vp, vp]
     L.kv_pool_set_attention_config.argtypes = [vp, i, i]
+    L.kv_pool_set_scorer_config.argtypes = [vp, i, i]
+    L.kv_pool_score_launch_info.argtypes = [vp, ip, ip, vp]
     _lib = L
     return L
 
@@ -225,6 +227,14 @@ class KVPool:
 
     def set_attention_config(self, grid_ctas=0, fast_path=0):
         _check("kv_pool_set_attention_config", lib().kv_pool_set_attention_config(self.handle, grid_ctas, fast_path))
+
+    def set_scorer_config(self, mode=0, tc_min_rows=0):
+        _check("kv_pool_set_scorer_config", lib().kv_pool_set_scorer_config(self.handle, mode, tc_min_rows))
+
+    def score_launch_info(self, stream=None):
+        n, u = C.c_int(), C.c_int()
+        _check("kv_pool_score_launch_info", lib().kv_pool_score_launch_info(self.handle, C.byref(n), C.byref(u), _stream(stream)))
+        return dict(n_rows=n.value, tc_units=u.value)
 
 
 class ScorerWeights:

@@ -286,6 +286,8 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->num_sms = sms;
   p->attn_grid = sms;
   p->fast_path = 1;
+  p->scorer_mode = 0;
+  p->scorer_tc_min_rows = 128;
   p->device = dev;
   p->lay = lay;
   char* m = static_cast<char*>(cfg->meta_storage);

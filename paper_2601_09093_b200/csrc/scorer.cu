@@ -4,13 +4,17 @@
 //   score_t = (1/n) sum_{i<=n} y_i^t               (Sec. 3.3)
 //
 // Only rows whose boundary flag is set are scored (Algorithm 1 runs the scorer when the new
-// token ends a step), so the launch is three kernels:
-//   compact : ascending list of boundary rows (block-wide prefix sum), NaN into the other rows
-//   mlp     : for a tile of listed rows and a slice of the m hidden units, the partial
-//             w2 . ReLU(W1 h + b1); hidden rows staged in shared memory as fp32, W1 rows streamed
-//             with 16-byte loads, fp32 accumulation, no rounding of the activations
-//   finish  : fixed-order sum of the slices, + b2, sigmoid, scatter to the row, then the
-//             per-trace (sum, count) update in ascending row order and the refreshed means.
+// token ends a step), so one launch is
+//   compact : ascending list of boundary rows (block-wide prefix sum), NaN into the other rows;
+//             it also decides, from the number of rows found, which first-layer kernel does the work
+//   mlp     : few rows (a decode step: about one boundary per 64 traces) - score_mlp_kernel, CUDA
+//             cores: for a tile of listed rows and a slice of the m hidden units the partial
+//             w2 . ReLU(W1 h + b1), hidden rows staged in shared memory as fp32, W1 rows streamed with
+//             16-byte loads;  many rows (batched scoring) - the tcgen05 kernel of scorer_tc.cu.
+//             Both accumulate in fp32 and never round the activations.
+//   rows    : fixed-order sum of the slices, + b2, sigmoid, scatter to the row
+//   traces  : a warp per trace folds that trace's new scores into (sum, count) in ascending row
+//             order and refreshes the mean.
 #include "step_internal.cuh"
 
 #include <math.h>
@@ -28,8 +32,11 @@ template <typename T> __device__ inline float cvt(T x);
 template <> __device__ inline float cvt<float>(float x) { return x; }
 template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 
+// tc_min_rows: 0 = the tensor-core kernel is not available for this launch; otherwise the smallest
+// number of boundary rows that goes to it.  m: hidden units; num_sms: for the tiling choice.
 __global__ void __launch_bounds__(kCompactThreads)
-score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float* __restrict__ step_scores) {
+score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float* __restrict__ step_scores,
+                     int tc_min_rows, int m, int num_sms) {
   __shared__ int s_warp[33];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int running = 0;
@@ -61,7 +68,23 @@ score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float*
     else if (i < M) step_scores[i] = __int_as_float(0x7fc00000);
     running += s_warp[32];
   }
-  if (threadIdx.x == 0) v.counters[C_SCORE_NB] = running;
+  if (threadIdx.x == 0) {
+    const int nb = running;
+    v.counters[C_SCORE_NB] = nb;
+    int N = 0;
+    if (tc_min_rows > 0 && nb >= tc_min_rows) {
+      // widest slice of hidden units per CTA (best reuse of the gathered rows) that still gives every SM
+      // an item; else the narrowest, which spreads a small launch over the most SMs
+      const int tiles = (nb + 127) / 128;
+      for (int cand = 256; cand >= 64; cand >>= 1) {
+        if (m % cand != 0 || m / cand > kSplits) continue;
+        N = cand;
+        if (tiles * (m / cand) >= num_sms) break;
+      }
+    }
+    v.counters[C_SCORE_TC] = N;
+    v.counters[C_SCORE_SLICES] = N ? m / N : kSplits;
+  }
 }
 
 // grid (kSplits, row tiles).  Dynamic shared memory: kRowTile * D floats.
@@ -71,6 +94,7 @@ score_mlp_kernel(DevViews v, const T* __restrict__ hidden, const T* __restrict__
                  const T* __restrict__ w2, int D, int m) {
   extern __shared__ float s_h[];                      // [kRowTile][D]
   __shared__ float s_part[kMlpWarps][kRowTile];
+  if (v.counters[C_SCORE_TC] != 0) return;            // this launch's rows belong to the tensor-core kernel
   const int nb = v.counters[C_SCORE_NB];
   const int r0 = blockIdx.y * kRowTile;
   if (r0 >= nb) return;
@@ -121,35 +145,55 @@ score_mlp_kernel(DevViews v, const T* __restrict__ hidden, const T* __restrict__
   }
 }
 
-__global__ void __launch_bounds__(1024)
-score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
-                    float unscored, float* __restrict__ step_scores) {
-  const int nb = v.counters[C_SCORE_NB];
-  for (int r = threadIdx.x; r < nb; r += blockDim.x) {
+// One thread per listed row: slices in fixed order, + b2, sigmoid, scatter.  The score is also left in
+// the row's first score_z slot for the per-trace fold.
+__global__ void __launch_bounds__(256)
+score_rows_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
+                  float* __restrict__ step_scores) {
+  const int nb = v.counters[C_SCORE_NB], ns = v.counters[C_SCORE_SLICES];
+  for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < nb; r += gridDim.x * blockDim.x) {
     float z = 0.f;
-    for (int s = 0; s < kSplits; ++s) z += v.score_z[(size_t)r * kSplits + s];
+    for (int s = 0; s < ns; ++s) z += v.score_z[(size_t)r * kSplits + s];
     z += b2;
     const float y = 1.f / (1.f + expf(-z));
-    step_scores[v.score_idx[r]] = y;
+    const int row = v.score_idx[r];
+    step_scores[row] = y;
     v.score_z[(size_t)r * kSplits] = y;
+    const int tr = row_trace ? row_trace[row] : row + row_base;
+    if (tr < 0 || tr >= g.max_traces) flag_error(v.counters, STEP_ERR_BAD_TRACE);   // names no trace of this pool
   }
-  __syncthreads();
-  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
-    float sum = v.score_sum[t];
-    int cnt = v.score_cnt[t];
-    for (int r = 0; r < nb; ++r) {
+}
+
+// A warp per trace: scan the listed rows 32 at a time and add this trace's scores one by one in
+// ascending row order (the order a serial loop over the rows would use), then refresh the mean.
+__global__ void __launch_bounds__(256)
+score_traces_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float unscored) {
+  const int nb = v.counters[C_SCORE_NB];
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= g.max_traces) return;
+  float sum = v.score_sum[t];
+  int cnt = v.score_cnt[t];
+  for (int base = 0; base < nb; base += 32) {
+    const int r = base + lane;
+    int tr = -1;
+    float y = 0.f;
+    if (r < nb) {
       const int row = v.score_idx[r];
-      const int tr = row_trace ? row_trace[row] : row + row_base;
-      if (tr == t) { sum += v.score_z[(size_t)r * kSplits]; ++cnt; }
+      tr = row_trace ? row_trace[row] : row + row_base;
+      y = v.score_z[(size_t)r * kSplits];
     }
+    unsigned hit = __ballot_sync(0xffffffffu, tr == t);
+    while (hit) {
+      const int src = __ffs(hit) - 1;
+      hit &= hit - 1;
+      sum += __shfl_sync(0xffffffffu, y, src);
+      ++cnt;
+    }
+  }
+  if (lane == 0) {
     v.score_sum[t] = sum; v.score_cnt[t] = cnt;
     v.trace_scores[t] = cnt > 0 ? sum / (float)cnt : unscored;
-  }
-  // rows that name no trace of this pool
-  for (int r = threadIdx.x; r < nb; r += blockDim.x) {
-    const int row = v.score_idx[r];
-    const int tr = row_trace ? row_trace[row] : row + row_base;
-    if (tr < 0 || tr >= g.max_traces) flag_error(v.counters, STEP_ERR_BAD_TRACE);
   }
 }
 
@@ -168,25 +212,57 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
   cudaStream_t s = (cudaStream_t)stream;
   Geo g = geo_of(pool);
   const size_t eb = w->dtype == STEP_BF16 ? 2 : 4;
+  const bool tc = pool->scorer_mode >= 0 && score_tc_supported(w, hidden);
+  const int tc_min_rows = !tc ? 0 : (pool->scorer_mode > 0 ? 1 : pool->scorer_tc_min_rows);
   for (int off = 0; off < M; off += pool->max_score_rows) {
     const int Mc = M - off < pool->max_score_rows ? M - off : pool->max_score_rows;
     const char* hid = (const char*)hidden + (size_t)off * w->D * eb;
     const int32_t* rt = row_trace ? row_trace + off : nullptr;
-    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, boundary_mask + off, Mc, step_scores_out + off);
-    dim3 grid(kSplits, (Mc + kRowTile - 1) / kRowTile);
-    if (w->dtype == STEP_BF16) {
-      auto kern = score_mlp_kernel<__nv_bfloat16>;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
-      kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const __nv_bfloat16*)hid, (const __nv_bfloat16*)w->W1,
-                                             (const __nv_bfloat16*)w->b1, (const __nv_bfloat16*)w->w2, w->D, w->m);
-    } else {
-      auto kern = score_mlp_kernel<float>;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
-      kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const float*)hid, (const float*)w->W1, (const float*)w->b1,
-                                             (const float*)w->w2, w->D, w->m);
+    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, boundary_mask + off, Mc, step_scores_out + off,
+                                                       tc_min_rows, w->m, pool->num_sms);
+    // the CUDA-core kernel only ever sees launches with fewer than tc_min_rows boundary rows
+    const int scalar_rows = tc_min_rows > 0 && tc_min_rows - 1 < Mc ? tc_min_rows - 1 : Mc;
+    if (scalar_rows > 0) {
+      dim3 grid(kSplits, (scalar_rows + kRowTile - 1) / kRowTile);
+      if (w->dtype == STEP_BF16) {
+        auto kern = score_mlp_kernel<__nv_bfloat16>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+        kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const __nv_bfloat16*)hid, (const __nv_bfloat16*)w->W1,
+                                               (const __nv_bfloat16*)w->b1, (const __nv_bfloat16*)w->w2, w->D, w->m);
+      } else {
+        auto kern = score_mlp_kernel<float>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+        kern<<<grid, kMlpWarps * 32, smem, s>>>(pool->v, (const float*)hid, (const float*)w->W1, (const float*)w->b1,
+                                               (const float*)w->w2, w->D, w->m);
+      }
+    }
+    if (tc_min_rows > 0 && Mc >= tc_min_rows) {
+      const int st = score_tc_launch(pool, hid, Mc, w, s);
+      if (st != STEP_OK) return st;
     }
     // row_trace == NULL means row i is trace i, counted from the start of the whole call
-    score_finish_kernel<<<1, 1024, 0, s>>>(pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off);
+    int row_ctas = (Mc + 255) / 256;
+    if (row_ctas > pool->num_sms * 4) row_ctas = pool->num_sms * 4;
+    score_rows_kernel<<<row_ctas, 256, 0, s>>>(pool->v, g, rt, off, w->b2, step_scores_out + off);
+    score_traces_kernel<<<(g.max_traces + 7) / 8, 256, 0, s>>>(pool->v, g, rt, off, pool->cfg.unscored_score);
   }
   return launch_ok();
+}
+
+extern "C" int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows) {
+  if (!pool || mode < -1 || mode > 1 || tc_min_rows < 0) return STEP_ERR_INVALID_ARG;
+  pool->scorer_mode = mode;
+  if (tc_min_rows > 0) pool->scorer_tc_min_rows = tc_min_rows;
+  return STEP_OK;
+}
+
+extern "C" int kv_pool_score_launch_info(step_pool* pool, int* n_rows, int* tc_units, void* stream) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t c[C_SCORE_SLICES + 1];
+  STEP_CUDA_OK(cudaMemcpyAsync(c, pool->v.counters, sizeof(c), cudaMemcpyDeviceToHost, s));
+  STEP_CUDA_OK(cudaStreamSynchronize(s));
+  if (n_rows) *n_rows = c[C_SCORE_NB];
+  if (tc_units) *tc_units = c[C_SCORE_TC];
+  return STEP_OK;
 }

@@ -1,0 +1,400 @@
+// Tensor-core form of the step scorer's first layer for launches with many boundary rows
+// (Sec. 3.1 "Model Architecture": y = sigmoid(w2 . ReLU(W1 h + b1) + b2)).
+//
+// For the listed rows r and a slice [n0, n0 + N) of the m hidden units one work item computes
+//     z_slice[r] = sum_{j in slice} w2[j] * ReLU(sum_k h[r][k] * W1[j][k] + b1[j])
+// as a 128 x N x D bf16 GEMM on the 5th-generation tensor cores with the whole second layer fused into
+// the read-out of the accumulator:
+//   * the accumulator (128 rows x N columns, fp32) lives in tensor memory; two of them (2 x 256 columns)
+//     let the read-out of one item overlap the products of the next;
+//   * A = the hidden rows named by the row list.  The rows are scattered in the caller's [M, D]
+//     array, so four warps gather them with 16-byte cp.async copies straight into the 128-byte-swizzled
+//     K-major arrangement the MMA unit reads (row r of a tile at (r / 8) * 1024 + (r % 8) * 128,
+//     16-byte chunk c stored at chunk c ^ (r % 8)); no compacted copy of the rows is ever made;
+//   * B = W1[n0 .. n0 + N, k .. k + 64): TMA tiled loads (one 64 x 64 box per 64 units, 128-byte
+//     swizzle) signalling the stage's mbarrier with their byte count;
+//   * one thread issues tcgen05.mma (M 128, N 64 | 128 | 256, K 16) four times per 64-wide k-chunk and
+//     commits the stage back to the producers;
+//   * four warps read the finished accumulator with tcgen05.ld - a thread owns one row, so
+//     + b1, ReLU, * w2 and the sum over the slice's units are plain per-thread fp32 arithmetic on
+//     un-rounded activations - and store one partial per (row, slice) for the finishing kernel.
+// The kernel is persistent (one CTA per SM, items handed out round-robin).  N is picked on the device
+// from the number of boundary rows so that small launches still spread over many SMs.
+// Every wait is bounded; a wait that runs out raises STEP_ERR_TIMEOUT and the CTA winds down,
+// releasing its tensor memory.
+#include "step_internal.cuh"
+
+#include <cuda.h>
+
+using namespace stepk;
+
+namespace {
+
+constexpr int kTileRows = 128;                    // UMMA M: rows of one item
+constexpr int kBK = 64;                           // bf16 elements per k-chunk (one 128-byte swizzle row)
+constexpr int kMaxN = 256;                        // UMMA N limit
+constexpr int kStages = 4;
+constexpr int kABytes = kTileRows * kBK * 2;      // 16 KiB
+constexpr int kBoxRows = 64;                      // hidden units per TMA box
+constexpr int kBoxBytes = kBoxRows * kBK * 2;     // 8 KiB
+constexpr int kBBytes = kMaxN * kBK * 2;          // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
+constexpr int kLag = 2;                           // gather groups a producer thread keeps in flight
+constexpr int kEpiWarps = 4, kGatherWarps = 4;
+constexpr int kWarpTma = kEpiWarps + kGatherWarps, kWarpMma = kWarpTma + 1;
+constexpr int kThreads = (kWarpMma + 1) * 32;     // 320
+constexpr int kTmemCols = 512;                    // two accumulators of up to 256 columns
+constexpr int kMaxUnits = 1024;                   // b1 / w2 staged in shared memory as fp32
+constexpr unsigned long long kWaitNs = 2000000000ull;
+constexpr unsigned long long kDrainNs = 100000000ull;
+
+struct TcArgs {
+  const __nv_bfloat16* hidden;
+  const __nv_bfloat16* b1;
+  const __nv_bfloat16* w2;
+  const int32_t* idx;
+  float* z;
+  int32_t* counters;
+  int D, m;
+};
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ inline void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ inline unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ inline bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_ns = kWaitNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > limit_ns) return false;
+  }
+}
+__device__ inline void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending> __device__ inline void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+}
+__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ inline void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ inline void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate.
+__device__ inline void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ inline void tc_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) stored with the
+// 128-byte swizzle: groups of 8 rows are 1024 bytes apart (stride byte offset), the leading byte offset is
+// unused by swizzled K-major layouts (1), descriptor version 1, layout type 2 = SWIZZLE_128B.
+__device__ inline uint64_t umma_desc_sw128(uint32_t smem_addr) {
+  const uint32_t lo = ((smem_addr >> 4) & 0x3FFFu) | (1u << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
+__device__ inline uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
+  // the launch decided on the device whether this kernel or the CUDA-core kernel scores its rows
+  const int N = a.counters[C_SCORE_TC];
+  if (N == 0) return;
+  const int nb = a.counters[C_SCORE_NB];
+  const int slices = a.m / N;
+  const int tiles = (nb + kTileRows - 1) / kTileRows;
+  const int items = tiles * slices;
+  const int KC = a.D / kBK;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles want 1024-byte alignment
+  unsigned char* sm = smem_raw + (base - raw);
+  float* s_b1 = reinterpret_cast<float*>(sm + kStages * kStageBytes);
+  float* s_w2 = s_b1 + kMaxUnits;
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_w2 + kMaxUnits);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  const uint32_t bar_full = smem_u32(s_bar), bar_empty = bar_full + 8 * kStages;
+  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 16;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, kGatherWarps + 1);            // one arrival per gather warp + the TMA thread
+      mbar_init(bar_empty + 8 * s, 1);                          // tcgen05.commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8 * b, 1);                          // tcgen05.commit
+      mbar_init(bar_tempty + 8 * b, kEpiWarps);                 // one arrival per read-out warp
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kWarpMma) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int j = threadIdx.x; j < a.m; j += kThreads) {
+    s_b1[j] = __bfloat162float(a.b1[j]);
+    s_w2[j] = __bfloat162float(a.w2[j]);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (warp < kEpiWarps) {
+    // ------------------------------------------------ read-out: second layer on the accumulator
+    int li = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x, ++li) {
+      const int tile = item / slices, slice = item - tile * slices, n0 = slice * N;
+      const int buf = li & 1;
+      if (*s_abort) break;
+      if (!mbar_wait_bounded(bar_tfull + 8 * buf, (li >> 1) & 1)) {
+        if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
+        *s_abort = 1;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kMaxN);
+      float z = 0.f;
+      for (int c0 = 0; c0 < N; c0 += 32) {
+        float v[32];
+        tc_ld32(taddr + c0, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) z = fmaf(s_w2[n0 + c0 + j], fmaxf(v[j] + s_b1[n0 + c0 + j], 0.f), z);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+      const int row = tile * kTileRows + warp * 32 + lane;
+      if (row < nb) a.z[(size_t)row * kScoreSplits + slice] = z;
+    }
+  } else if (warp < kWarpTma) {
+    // ------------------------------------------------ gather of the listed hidden rows into A
+    const int tg = threadIdx.x - kEpiWarps * 32;                // 0 .. 127
+    const int c = tg & 7, rb = tg >> 3;                         // 16-byte chunk of the row; rows rb + 16 i
+    const uint32_t dst0 = base + (uint32_t)((rb >> 3) * 1024 + (rb & 7) * 128 + ((c ^ (rb & 7)) << 4));
+    const uint32_t my_full = bar_full;
+    int it = 0, signalled = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+      const int tile = item / slices;
+      const __nv_bfloat16* src[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        int gr = tile * kTileRows + rb + 16 * i;
+        if (gr >= nb) gr = nb - 1;                              // rows past the list re-read its last row; never stored
+        src[i] = a.hidden + (size_t)a.idx[gr] * a.D + c * 8;
+      }
+      for (int kc = 0; kc < KC; ++kc, ++it) {
+        const int s = it % kStages;
+        if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
+        const uint32_t dst = dst0 + (uint32_t)(s * kStageBytes);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cp_async16(dst + i * 2048, src[i] + kc * kBK);
+        cp_async_commit();
+        if (it >= kLag) {
+          cp_async_wait<kLag>();                                // chunk it - kLag of this thread has landed
+          fence_async_smem();                                   // ... and is visible to the tensor core's reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive(my_full + 8 * ((it - kLag) % kStages));
+          ++signalled;
+        }
+      }
+    }
+    cp_async_wait<0>();
+    fence_async_smem();
+    __syncwarp();
+    if (ok) {
+      for (; signalled < it; ++signalled)
+        if (lane == 0) mbar_arrive(my_full + 8 * (signalled % kStages));
+    } else {
+      if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
+      *s_abort = 1;
+    }
+  } else if (warp == kWarpTma) {
+    // ------------------------------------------------ TMA loads of the W1 slice into B
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      const int boxes = N / kBoxRows;
+      for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+        const int n0 = (item % slices) * N;
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % kStages;
+          if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
+          const uint32_t bar = bar_full + 8 * s;
+          mbar_expect_tx(bar, (uint32_t)(boxes * kBoxBytes));
+          const uint32_t dst = base + (uint32_t)(s * kStageBytes + kABytes);
+          for (int j = 0; j < boxes; ++j) tma_load_2d(dst + j * kBoxBytes, &map_w1, kc * kBK, n0 + j * kBoxRows, bar);
+        }
+      }
+      if (!ok) {
+        flag_error(a.counters, STEP_ERR_TIMEOUT);
+        *s_abort = 1;
+        // loads already issued still target this CTA's shared memory: give them a moment to land
+        for (int s = 0; s < kStages; ++s) {
+          mbar_wait_bounded(bar_full + 8 * s, 0, kDrainNs);
+          mbar_wait_bounded(bar_full + 8 * s, 1, kDrainNs);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ MMA issue
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(N);
+      int it = 0, li = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++li) {
+        const int buf = li & 1;
+        if (*s_abort || !mbar_wait_bounded(bar_tempty + 8 * buf, ((li >> 1) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kMaxN);
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % kStages;
+          if (*s_abort || !mbar_wait_bounded(bar_full + 8 * s, (it / kStages) & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes));
+          const uint64_t bdesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + kABytes));
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk)                  // 16 bf16 = 32 bytes further along the swizzled row
+            tc_mma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | kk) != 0);
+          tc_commit(bar_empty + 8 * s);                         // the stage is free once these products have read it
+        }
+        if (ok) tc_commit(bar_tfull + 8 * buf);                 // the accumulator is complete
+      }
+      if (!ok) {
+        flag_error(a.counters, STEP_ERR_TIMEOUT);
+        *s_abort = 1;
+      }
+    }
+    __syncwarp();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kWarpMma) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 2 * kMaxUnits * sizeof(float) +
+                              (2 * kStages + 4) * sizeof(uint64_t) + 16;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    tried = true;
+  }
+  return fn;
+}
+
+}  // namespace
+
+namespace stepk {
+
+bool score_tc_supported(const scorer_weights* w, const void* hidden) {
+  if (w->dtype != STEP_BF16) return false;
+  if (w->D < kBK || w->D % kBK != 0) return false;                       // whole 64-wide k-chunks
+  if (w->m < kBoxRows || w->m % kBoxRows != 0 || w->m > kMaxUnits) return false;
+  if (w->m / kMaxN > kScoreSplits) return false;
+  if (((uintptr_t)w->W1 | (uintptr_t)hidden) & 15) return false;         // 16-byte copies and TMA base
+  return encode_tiled_fn() != nullptr;
+}
+
+int score_tc_launch(const step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return STEP_ERR_CUDA;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)w->D, (cuuint64_t)w->m};       // innermost first
+  const cuuint64_t strides[1] = {(cuuint64_t)w->D * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kBoxRows};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w->W1), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return STEP_ERR_CUDA;
+  if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+    return STEP_ERR_CUDA;
+  TcArgs a;
+  a.hidden = (const __nv_bfloat16*)hidden;
+  a.b1 = (const __nv_bfloat16*)w->b1; a.w2 = (const __nv_bfloat16*)w->w2;
+  a.idx = pool->v.score_idx; a.z = pool->v.score_z; a.counters = pool->v.counters;
+  a.D = w->D; a.m = w->m;
+  long long max_items = (long long)((Mc + kTileRows - 1) / kTileRows) * (w->m / kBoxRows);
+  int grid = pool->num_sms;
+  if (max_items < grid) grid = (int)max_items;
+  if (grid < 1) grid = 1;
+  score_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(map, a);
+  return launch_ok();
+}
+
+}  // namespace stepk

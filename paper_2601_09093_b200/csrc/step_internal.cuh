@@ -23,7 +23,11 @@ constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream p
 constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
 constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
 
-enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4, C_NUM = 64 };
+// C_SCORE_TC: 0 = the launch's boundary rows go through the CUDA-core MLP kernel; otherwise the
+// number of hidden units (UMMA N) each CTA of the tensor-core kernel covers.  C_SCORE_SLICES:
+// how many partial sums per row the MLP kernels leave in score_z.
+enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4,
+               C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_NUM = 64 };
 
 struct MetaLayout {
   size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;
@@ -55,6 +59,8 @@ struct step_pool {
   int num_sms;
   int attn_grid;      // CTAs of the tensor-core attention launch
   int fast_path;      // 1 allowed, -1 forced off
+  int scorer_mode;    // 0: tensor-core MLP for launches with >= scorer_tc_min_rows boundary rows; 1: always; -1: never
+  int scorer_tc_min_rows;
   int device;
   stepk::MetaLayout lay;
   stepk::DevViews v;
@@ -98,5 +104,12 @@ __device__ inline void flag_error(int32_t* counters, int code) {
   } while (0)
 
 inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? STEP_OK : STEP_ERR_CUDA; }
+
+// ---- tensor-core scorer (scorer_tc.cu)
+// True if the tcgen05 kernel covers this scorer shape and these pointers.
+bool score_tc_supported(const scorer_weights* w, const void* hidden);
+// Launches the persistent kernel for a chunk of Mc candidate rows (at most one CTA per SM); it reads
+// C_SCORE_NB / C_SCORE_TC on the device and returns at once when C_SCORE_TC is 0.
+int score_tc_launch(const step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s);
 
 }  // namespace stepk

@@ -204,9 +204,16 @@ def test_bad_block_table_is_flagged():
 
 
 # ------------------------------------------------------------------ scorer
-def _scorer_case(cfg, M, density, row_trace=None, bias=0.05, max_traces=None, max_score_rows=0):
+def _scorer_case(cfg, M, density, row_trace=None, bias=0.05, max_traces=None, max_score_rows=0, mode=0,
+                 tc_min_rows=0, expect_tc=None, sample=0):
+    """score_steps against the oracle.  mode / tc_min_rows pick the first-layer kernel (0 = the library's
+    own choice); expect_tc checks which one ran (hidden units per CTA of the tensor-core kernel, 0 = the
+    CUDA-core kernel).  sample > 0: only that many boundary rows (spread over the list, ends included) are
+    given to the oracle - for launches too large for it; the running means are then checked against the
+    GPU's own step scores only."""
     T = max_traces or cfg.n_traces
     pool = H.make_pool(cfg, 8, 4, T, max_score_rows=max_score_rows)
+    pool.set_scorer_config(mode, tc_min_rows)
     (W1b, W1x), (b1b, b1x), (w2b, w2x), b2 = W.scorer_weights(cfg, bias_std=bias)
     wts = B.ScorerWeights(H.to_device(W1b, cfg.dtype), H.to_device(b1b, cfg.dtype), H.to_device(w2b, cfg.dtype), b2,
                           H.step_dtype(cfg))
@@ -214,19 +221,32 @@ def _scorer_case(cfg, M, density, row_trace=None, bias=0.05, max_traces=None, ma
     mask = W.boundary_mask(cfg, M, density=density)
     rt_dev = None if row_trace is None else torch.from_numpy(row_trace.astype(np.int32)).cuda()
     got = pool.score_steps(H.to_device(hb, cfg.dtype), torch.from_numpy(mask).cuda(), rt_dev, wts)
-    want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+    if expect_tc is not None:
+        info = pool.score_launch_info()
+        assert info["tc_units"] == expect_tc, info
     g = got.cpu().numpy()
     assert np.isnan(g[mask == 0]).all()
-    if mask.any():
-        assert np.abs(g[mask == 1] - want[mask == 1]).max() <= SCORE_TOL
+    assert not np.isnan(g[mask == 1]).any()
+    if sample:
+        rows = np.flatnonzero(mask)
+        pick = rows[np.unique(np.linspace(0, len(rows) - 1, sample).astype(np.int64))]
+        W1d, b1d, w2d = W1x.astype(np.float64), b1x.astype(np.float64), w2x.astype(np.float64)
+        want_s = np.array([OS.step_score(hx[i], W1d, b1d, w2d, b2) for i in pick])
+        assert np.abs(g[pick] - want_s).max() <= SCORE_TOL
+        want = None
+    else:
+        want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+        if mask.any():
+            assert np.abs(g[mask == 1] - want[mask == 1]).max() <= SCORE_TOL
     ts = OS.TraceScores(T)
     ts.update(g, mask, row_trace)                       # running means from the GPU's own step scores
     v = pool.views()
-    np.testing.assert_allclose(v["trace_scores"].cpu().numpy(), ts.scores(), atol=1e-6)
+    np.testing.assert_allclose(v["trace_scores"].cpu().numpy(), ts.scores(), atol=2e-6 if M <= 3000 else 1e-5)
     np.testing.assert_array_equal(v["score_cnt"].cpu().numpy(), ts.cnt)
-    ts2 = OS.TraceScores(T)
-    ts2.update(want, mask, row_trace)                   # and within tolerance of the all-oracle means
-    assert np.abs(v["trace_scores"].cpu().numpy() - ts2.scores()).max() <= SCORE_TOL
+    if want is not None:
+        ts2 = OS.TraceScores(T)
+        ts2.update(want, mask, row_trace)               # and within tolerance of the all-oracle means
+        assert np.abs(v["trace_scores"].cpu().numpy() - ts2.scores()).max() <= SCORE_TOL
     assert pool.last_error() == (0, 0)
     return pool, wts, g, mask
 
@@ -253,7 +273,47 @@ def test_scorer_batched_rows_with_row_trace_and_chunking():
 
 
 def test_scorer_c4_shape():
-    _scorer_case(W.C4, 128, 0.1)
+    _scorer_case(W.C4, 128, 0.1, expect_tc=0)
+
+
+# ---- the tensor-core first layer (tcgen05): same rows, same tolerance
+def test_scorer_tensor_core_partial_tile():
+    """Fewer rows than one 128-row tile, forced onto the tensor cores (narrowest slices)."""
+    _scorer_case(W.C1, 64, 1.0 / 8, mode=1, expect_tc=64)
+    _scorer_case(W.C1, 64, 1.0, mode=1, expect_tc=64)
+    _scorer_case(W.C1, 64, 0.0, mode=1, expect_tc=0)              # no boundary row: nothing to do
+
+
+def test_scorer_tensor_core_c4_shape():
+    """m = 1024, D = 5120: sixteen 64-unit slices, 80 k-chunks."""
+    _scorer_case(W.C4, 128, 0.5, mode=1, expect_tc=64)
+
+
+def test_scorer_tensor_core_ragged_tiles_with_row_trace():
+    """Several tiles and a ragged last one, rows scattered over the input by the mask, many rows per trace."""
+    cfg = W.C1
+    M = 64 * 40 + 13
+    rt = (np.arange(M) % 64).astype(np.int32)
+    _scorer_case(cfg, M, 1.0 / 4, row_trace=rt, max_score_rows=M, expect_tc=64)       # ~640 rows: library's choice
+    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M, tc_min_rows=100, expect_tc=64)
+
+
+def test_scorer_picks_the_cuda_core_kernel_below_the_row_threshold():
+    rt = (np.arange(512) % 64).astype(np.int32)
+    _scorer_case(W.C1, 512, 1.0 / 8, row_trace=rt, max_score_rows=512, expect_tc=0)         # ~64 rows < 128
+    _scorer_case(W.C1, 512, 1.0, row_trace=rt, max_score_rows=512, mode=-1, expect_tc=0)    # forced off
+
+
+@pytest.mark.parametrize("rows,units", [(4800, 128), (9600, 256)])
+def test_scorer_tensor_core_wide_slices_sampled(rows, units):
+    """Launches large enough that the device picks 128- and 256-unit slices (several items per CTA, both
+    accumulators in use).  The oracle scores a sample of rows; the CUDA-core kernel, itself checked against
+    the oracle above, cross-checks every row."""
+    cfg = W.C1
+    rt = (np.arange(rows) % 64).astype(np.int32)
+    _, _, g_tc, mask = _scorer_case(cfg, rows, 1.0, row_trace=rt, max_score_rows=rows, expect_tc=units, sample=96)
+    _, _, g_cc, _ = _scorer_case(cfg, rows, 1.0, row_trace=rt, max_score_rows=rows, mode=-1, expect_tc=0, sample=8)
+    assert np.abs(g_tc - g_cc).max() <= 1e-4
 
 
 def test_scorer_running_mean_accumulates_across_calls():
