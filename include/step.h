@@ -200,7 +200,8 @@ int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path);
  * (D a multiple of 64, m a multiple of 64 and <= 1024, 16-byte aligned W1 and hidden): mode 0 (default)
  * sends a launch to the tensor cores when it has at least tc_min_rows boundary rows (the count is taken
  * on the device) and to the CUDA-core kernel otherwise; mode 1 always uses the tensor cores, mode -1 never.
- * tc_min_rows = 0 keeps the current value (default 128). */
+ * tc_min_rows = 0 keeps the current value (default 1: measured faster than the CUDA-core kernel from the
+ * first row on; fp32 scorers and other shapes always take the CUDA-core kernel). */
 int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows);
 /* What the most recent score_steps launch did (of its last chunk, if M exceeded max_score_rows):
  * *n_rows = boundary rows it found, *tc_units = hidden units per CTA of the tensor-core kernel, or 0 if

@@ -49,6 +49,7 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.prune_off = take((T + 1) * 4);
   l.score_idx = take(rows * 4);
   l.score_z = take(rows * kScoreSplits * 4);
+  l.score_part = take((rows + kScoreFoldRows - 1) / kScoreFoldRows * T * 8);
   l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
   l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
   l.total = off;
@@ -287,7 +288,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->attn_grid = sms;
   p->fast_path = 1;
   p->scorer_mode = 0;
-  p->scorer_tc_min_rows = 128;
+  p->scorer_tc_min_rows = 1;
   p->device = dev;
   p->lay = lay;
   char* m = static_cast<char*>(cfg->meta_storage);
@@ -300,6 +301,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.append_base = (int32_t*)(m + lay.append_base); v.prune_rank = (int32_t*)(m + lay.prune_rank);
   v.prune_list = (int32_t*)(m + lay.prune_list); v.prune_off = (int32_t*)(m + lay.prune_off);
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
+  v.score_part = (float2*)(m + lay.score_part);
   v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o);
   int st = kv_pool_reset(p, nullptr);
   if (st == STEP_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = STEP_ERR_CUDA;

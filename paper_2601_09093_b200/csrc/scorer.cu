@@ -12,9 +12,9 @@
 //             w2 . ReLU(W1 h + b1), hidden rows staged in shared memory as fp32, W1 rows streamed with
 //             16-byte loads;  many rows (batched scoring) - the tcgen05 kernel of scorer_tc.cu.
 //             Both accumulate in fp32 and never round the activations.
-//   rows    : fixed-order sum of the slices, + b2, sigmoid, scatter to the row
-//   traces  : a warp per trace folds that trace's new scores into (sum, count) in ascending row
-//             order and refreshes the mean.
+//   finish  : fixed-order sum of the slices, + b2, sigmoid, scatter to the row; then every trace's new
+//             scores are folded into its (sum, count) in ascending row order (per 512-row CTA, the
+//             CTA partials in CTA order) and the mean is refreshed.
 #include "step_internal.cuh"
 
 #include <math.h>
@@ -34,16 +34,24 @@ template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return
 
 // tc_min_rows: 0 = the tensor-core kernel is not available for this launch; otherwise the smallest
 // number of boundary rows that goes to it.  m: hidden units; num_sms: for the tiling choice.
+// One CTA; a thread looks at kRowsPerThread consecutive rows per pass.
+constexpr int kRowsPerThread = 8;
+
 __global__ void __launch_bounds__(kCompactThreads)
 score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float* __restrict__ step_scores,
                      int tc_min_rows, int m, int num_sms) {
   __shared__ int s_warp[33];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float nan = __int_as_float(0x7fc00000);
   int running = 0;
-  for (int base = 0; base < M; base += blockDim.x) {
-    const int i = base + threadIdx.x;
-    const int f = i < M ? (mask[i] != 0) : 0;
-    int incl = f;
+  for (int base = 0; base < M; base += blockDim.x * kRowsPerThread) {
+    const int i0 = base + threadIdx.x * kRowsPerThread;
+    unsigned flags = 0;
+#pragma unroll
+    for (int j = 0; j < kRowsPerThread; ++j)
+      if (i0 + j < M && mask[i0 + j] != 0) flags |= 1u << j;
+    const int mine = __popc(flags);
+    int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int x = __shfl_up_sync(0xffffffffu, incl, o);
@@ -64,13 +72,18 @@ score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float*
       if (lane == 31) s_warp[32] = wi;
     }
     __syncthreads();
-    if (f) v.score_idx[running + s_warp[warp] + incl - 1] = i;
-    else if (i < M) step_scores[i] = __int_as_float(0x7fc00000);
+    int at = running + s_warp[warp] + incl - mine;
+#pragma unroll
+    for (int j = 0; j < kRowsPerThread; ++j) {
+      if (flags & (1u << j)) v.score_idx[at++] = i0 + j;
+      else if (i0 + j < M) step_scores[i0 + j] = nan;
+    }
     running += s_warp[32];
   }
   if (threadIdx.x == 0) {
     const int nb = running;
     v.counters[C_SCORE_NB] = nb;
+    v.counters[C_SCORE_TICKET] = 0;
     int N = 0;
     if (tc_min_rows > 0 && nb >= tc_min_rows) {
       // widest slice of hidden units per CTA (best reuse of the gathered rows) that still gives every SM
@@ -145,53 +158,57 @@ score_mlp_kernel(DevViews v, const T* __restrict__ hidden, const T* __restrict__
   }
 }
 
-// One thread per listed row: slices in fixed order, + b2, sigmoid, scatter.  The score is also left in
-// the row's first score_z slot for the per-trace fold.
+// Finishing kernel.  CTA c owns listed rows [c * kScoreFoldRows, ...):
+//   1. per row: slices in fixed order, + b2, sigmoid, scatter to step_scores;
+//   2. per trace: the sum and count of this CTA's rows that belong to it, rows in ascending order
+//      (a thread per trace walks the CTA's rows in shared memory), written as one partial;
+//   3. the CTA that finishes last adds the partials of every trace in CTA order to the trace's running
+//      (sum, count) and refreshes the mean - a fixed order, whichever CTA happens to be last.
 __global__ void __launch_bounds__(256)
-score_rows_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
-                  float* __restrict__ step_scores) {
+score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
+                    float unscored, float* __restrict__ step_scores) {
+  __shared__ float s_y[kScoreFoldRows];
+  __shared__ int s_tr[kScoreFoldRows];
+  __shared__ int s_last;
   const int nb = v.counters[C_SCORE_NB], ns = v.counters[C_SCORE_SLICES];
-  for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < nb; r += gridDim.x * blockDim.x) {
+  const int chunks = (nb + kScoreFoldRows - 1) / kScoreFoldRows;
+  const int c = blockIdx.x;
+  if (c >= chunks) return;
+  const int r0 = c * kScoreFoldRows, n = min(kScoreFoldRows, nb - r0);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int r = r0 + i;
     float z = 0.f;
     for (int s = 0; s < ns; ++s) z += v.score_z[(size_t)r * kSplits + s];
     z += b2;
     const float y = 1.f / (1.f + expf(-z));
     const int row = v.score_idx[r];
     step_scores[row] = y;
-    v.score_z[(size_t)r * kSplits] = y;
     const int tr = row_trace ? row_trace[row] : row + row_base;
     if (tr < 0 || tr >= g.max_traces) flag_error(v.counters, STEP_ERR_BAD_TRACE);   // names no trace of this pool
+    s_y[i] = y; s_tr[i] = tr;
   }
-}
-
-// A warp per trace: scan the listed rows 32 at a time and add this trace's scores one by one in
-// ascending row order (the order a serial loop over the rows would use), then refresh the mean.
-__global__ void __launch_bounds__(256)
-score_traces_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float unscored) {
-  const int nb = v.counters[C_SCORE_NB];
-  const int lane = threadIdx.x & 31;
-  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (t >= g.max_traces) return;
-  float sum = v.score_sum[t];
-  int cnt = v.score_cnt[t];
-  for (int base = 0; base < nb; base += 32) {
-    const int r = base + lane;
-    int tr = -1;
-    float y = 0.f;
-    if (r < nb) {
-      const int row = v.score_idx[r];
-      tr = row_trace ? row_trace[row] : row + row_base;
-      y = v.score_z[(size_t)r * kSplits];
-    }
-    unsigned hit = __ballot_sync(0xffffffffu, tr == t);
-    while (hit) {
-      const int src = __ffs(hit) - 1;
-      hit &= hit - 1;
-      sum += __shfl_sync(0xffffffffu, y, src);
-      ++cnt;
-    }
+  __syncthreads();
+  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
+    float sum = 0.f;
+    int cnt = 0;
+    for (int i = 0; i < n; ++i)
+      if (s_tr[i] == t) { sum += s_y[i]; ++cnt; }
+    v.score_part[(size_t)c * g.max_traces + t] = make_float2(sum, __int_as_float(cnt));
   }
-  if (lane == 0) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&v.counters[C_SCORE_TICKET], 1) == chunks - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
+    float sum = v.score_sum[t];
+    int cnt = v.score_cnt[t];
+    for (int k = 0; k < chunks; ++k) {
+      const float2 p = __ldcg(&v.score_part[(size_t)k * g.max_traces + t]);
+      const int pc = __float_as_int(p.y);
+      if (pc) { sum += p.x; cnt += pc; }
+    }
     v.score_sum[t] = sum; v.score_cnt[t] = cnt;
     v.trace_scores[t] = cnt > 0 ? sum / (float)cnt : unscored;
   }
@@ -241,10 +258,8 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
       if (st != STEP_OK) return st;
     }
     // row_trace == NULL means row i is trace i, counted from the start of the whole call
-    int row_ctas = (Mc + 255) / 256;
-    if (row_ctas > pool->num_sms * 4) row_ctas = pool->num_sms * 4;
-    score_rows_kernel<<<row_ctas, 256, 0, s>>>(pool->v, g, rt, off, w->b2, step_scores_out + off);
-    score_traces_kernel<<<(g.max_traces + 7) / 8, 256, 0, s>>>(pool->v, g, rt, off, pool->cfg.unscored_score);
+    score_finish_kernel<<<(Mc + kScoreFoldRows - 1) / kScoreFoldRows, 256, 0, s>>>(
+        pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off);
   }
   return launch_ok();
 }

@@ -39,7 +39,7 @@ constexpr int kBoxRows = 64;                      // hidden units per TMA box
 constexpr int kBoxBytes = kBoxRows * kBK * 2;     // 8 KiB
 constexpr int kBBytes = kMaxN * kBK * 2;          // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
-constexpr int kLag = 2;                           // gather groups a producer thread keeps in flight
+constexpr int kLag = 3;                           // gather groups a producer thread keeps in flight
 constexpr int kEpiWarps = 4, kGatherWarps = 4;
 constexpr int kWarpTma = kEpiWarps + kGatherWarps, kWarpMma = kWarpTma + 1;
 constexpr int kThreads = (kWarpMma + 1) * 32;     // 320
@@ -143,6 +143,11 @@ __device__ inline uint64_t umma_desc_sw128(uint32_t smem_addr) {
   const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
   return ((uint64_t)hi << 32) | lo;
 }
+// The k-chunk an item starts its reduction at.  Every item walks all D / 64 chunks once, cyclically; starting
+// them at different chunks keeps the CTAs that run side by side from all asking for the same few lines of
+// W1 (and the same byte offset of every hidden row) at the same moment.
+__device__ inline int first_chunk(int item, int KC) { return (int)(((unsigned)item * 7u) % (unsigned)KC); }
+
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
 __device__ inline uint32_t umma_idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
@@ -242,12 +247,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
         if (gr >= nb) gr = nb - 1;                              // rows past the list re-read its last row; never stored
         src[i] = a.hidden + (size_t)a.idx[gr] * a.D + c * 8;
       }
+      int kr = first_chunk(item, KC);
       for (int kc = 0; kc < KC; ++kc, ++it) {
         const int s = it % kStages;
         if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
         const uint32_t dst = dst0 + (uint32_t)(s * kStageBytes);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16(dst + i * 2048, src[i] + kc * kBK);
+        for (int i = 0; i < 8; ++i) cp_async16(dst + i * 2048, src[i] + kr * kBK);
+        if (++kr == KC) kr = 0;
         cp_async_commit();
         if (it >= kLag) {
           cp_async_wait<kLag>();                                // chunk it - kLag of this thread has landed
@@ -276,13 +283,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       const int boxes = N / kBoxRows;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
         const int n0 = (item % slices) * N;
+        int kr = first_chunk(item, KC);
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % kStages;
           if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
           const uint32_t bar = bar_full + 8 * s;
           mbar_expect_tx(bar, (uint32_t)(boxes * kBoxBytes));
           const uint32_t dst = base + (uint32_t)(s * kStageBytes + kABytes);
-          for (int j = 0; j < boxes; ++j) tma_load_2d(dst + j * kBoxBytes, &map_w1, kc * kBK, n0 + j * kBoxRows, bar);
+          for (int j = 0; j < boxes; ++j) tma_load_2d(dst + j * kBoxBytes, &map_w1, kr * kBK, n0 + j * kBoxRows, bar);
+          if (++kr == KC) kr = 0;
         }
       }
       if (!ok) {

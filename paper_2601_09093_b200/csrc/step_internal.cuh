@@ -22,18 +22,19 @@ namespace stepk {
 constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream partitions of one launch
 constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
 constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
+constexpr int kScoreFoldRows = 512;    // listed rows one CTA of the scorer's finishing kernel folds into per-trace partials
 
 // C_SCORE_TC: 0 = the launch's boundary rows go through the CUDA-core MLP kernel; otherwise the
 // number of hidden units (UMMA N) each CTA of the tensor-core kernel covers.  C_SCORE_SLICES:
 // how many partial sums per row the MLP kernels leave in score_z.
 enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4,
-               C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_NUM = 64 };
+               C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_SCORE_TICKET = 7, C_NUM = 64 };
 
 struct MetaLayout {
   size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;
   size_t refcount, free_list, claim, counters;
   size_t append_base, prune_rank, prune_list, prune_off;
-  size_t score_idx, score_z;
+  size_t score_idx, score_z, score_part;
   size_t attn_ml, attn_o;
   size_t total;
 };
@@ -43,7 +44,7 @@ struct DevViews {
   float* score_sum; int32_t* score_cnt; float* trace_scores;
   int32_t* refcount; int32_t* free_list; int32_t* claim; int32_t* counters;
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
-  int32_t* score_idx; float* score_z;
+  int32_t* score_idx; float* score_z; float2* score_part;
   float* attn_ml; float* attn_o;
 };
 

@@ -255,25 +255,35 @@ def test_c0_scorer_fp32():
     _scorer_case(W.C0, 8, 1.0, bias=0.0)
 
 
-def test_scorer_bf16_decode_shape():
-    _scorer_case(W.C1, 64, 1.0 / 8)
+# mode -1: the CUDA-core first layer; mode 0: the library's choice (tensor cores for these shapes)
+@pytest.mark.parametrize("mode", [-1, 0])
+def test_scorer_bf16_decode_shape(mode):
+    _scorer_case(W.C1, 64, 1.0 / 8, mode=mode, expect_tc=0 if mode < 0 else 64)
 
 
-def test_scorer_bf16_all_and_none_boundaries():
-    _scorer_case(W.C1, 64, 1.0)
-    _scorer_case(W.C1, 64, 0.0)
+@pytest.mark.parametrize("mode", [-1, 0])
+def test_scorer_bf16_all_and_none_boundaries(mode):
+    _scorer_case(W.C1, 64, 1.0, mode=mode)
+    _scorer_case(W.C1, 64, 0.0, mode=mode, expect_tc=0)
 
 
-def test_scorer_batched_rows_with_row_trace_and_chunking():
+@pytest.mark.parametrize("mode", [-1, 0])
+def test_scorer_batched_rows_with_row_trace_and_chunking(mode):
     cfg = W.C1
     M = 64 * 40 + 13
     rt = (np.arange(M) % 64).astype(np.int32)
-    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M)
-    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=1000)    # several launches
+    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M, mode=mode)
+    _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=1000, mode=mode)    # several launches
 
 
-def test_scorer_c4_shape():
-    _scorer_case(W.C4, 128, 0.1, expect_tc=0)
+def test_scorer_c4_shape_cuda_cores():
+    _scorer_case(W.C4, 128, 0.1, mode=-1, expect_tc=0)
+
+
+def test_scorer_odd_shapes_take_the_cuda_core_kernel():
+    """D not a multiple of 64 / m not a multiple of 64: outside the tensor-core kernel's shapes."""
+    _scorer_case(W.scaled(W.C1, scorer_D=1000, scorer_m=96), 64, 0.5, mode=0, expect_tc=0)
+    _scorer_case(W.scaled(W.C1, scorer_D=1024, scorer_m=96), 64, 0.5, mode=1, expect_tc=0)
 
 
 # ---- the tensor-core first layer (tcgen05): same rows, same tolerance
@@ -294,13 +304,13 @@ def test_scorer_tensor_core_ragged_tiles_with_row_trace():
     cfg = W.C1
     M = 64 * 40 + 13
     rt = (np.arange(M) % 64).astype(np.int32)
-    _scorer_case(cfg, M, 1.0 / 4, row_trace=rt, max_score_rows=M, expect_tc=64)       # ~640 rows: library's choice
+    _scorer_case(cfg, M, 1.0 / 4, row_trace=rt, max_score_rows=M, expect_tc=64)       # ~640 rows
     _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M, tc_min_rows=100, expect_tc=64)
 
 
 def test_scorer_picks_the_cuda_core_kernel_below_the_row_threshold():
     rt = (np.arange(512) % 64).astype(np.int32)
-    _scorer_case(W.C1, 512, 1.0 / 8, row_trace=rt, max_score_rows=512, expect_tc=0)         # ~64 rows < 128
+    _scorer_case(W.C1, 512, 1.0 / 8, row_trace=rt, max_score_rows=512, tc_min_rows=128, expect_tc=0)   # ~64 rows
     _scorer_case(W.C1, 512, 1.0, row_trace=rt, max_score_rows=512, mode=-1, expect_tc=0)    # forced off
 
 
