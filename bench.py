@@ -38,7 +38,11 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer"])
+    ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
+    ap.add_argument("--scorer-density", type=float, default=1.0, help="fraction of those rows that end a step")
+    ap.add_argument("--scorer-shape", default="c1", choices=["c1", "c4"])
+    ap.add_argument("--no-aux", action="store_true", help="skip the scorer / prune-cycle measurements after the timed steps")
     ap.add_argument("--num-blocks", type=int, default=0, help="override the pool size (blocks)")
     ap.add_argument("--grid", type=int, default=0, help="CTAs of the attention launch (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -46,13 +50,21 @@ def parse_args():
     return ap.parse_args()
 
 
-def measured_peaks():
+# DRAM bytes moved per algorithmic byte by attn_mma_kernel: dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture on the one-layer 64-trace workload (2.6895 GB + 6.56 MB against 2.665 GB algorithmic; the summary is
+# profiles/attn_mma_kernel_C1_ncu_full.md).  The kernel streams every page once, so traffic grows in proportion to
+# the algorithmic bytes and the larger workloads scale this figure.  Set to None when the kernel changes.
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (2.6895e9 + 6.56e6) / 2.665e9
+
+
+def measured_peaks(key="hbm_gbs", fallback=6650.0):
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        if key in d:
+            return float(d[key]), "measured"
+    return fallback, "fallback"
 
 
 class ClockSampler:
@@ -117,7 +129,8 @@ def workload_plan(name, num_blocks_override, steps_total, free_bytes=None):
         if p0 < 1:
             raise SystemExit("pool too small for the memory-saturated workload")
         suffix = np.full(cfg.n_traces, p0 * cfg.page_size, dtype=np.int64)
-        max_pages = shared + p0 + margin_pages + 2
+        # the prune cycles that follow the timed steps grow the survivors until 2 traces share the pool
+        max_pages = max(shared + p0 + margin_pages + 2, shared + limit // 4 + 64)
         return cfg, suffix, nb, max_pages, cfg.num_layers
     cfg = {"c1": W.C1, "c2": W.C2, "c4": W.C4}[name]
     suffix = W.suffix_lengths(cfg)
@@ -164,8 +177,9 @@ def run_ours(args):
     if cfg.shuffle_pages:
         H.shuffle_free_list(pool, cfg.seed + rank)
     t_fill = time.time()
+    append_log = []                                    # every append_kv call, for the oracle's replay of the prune cycles
     ids = H.fill_random_device(pool, cfg_pool, suffix, seed=cfg.seed + 7919 * rank,
-                               chunk_tokens=max(16, (1 << 28) // (T * cfg_pool.bytes_per_token)))
+                               chunk_tokens=max(16, (1 << 28) // (T * cfg_pool.bytes_per_token)), log=append_log)
     torch.cuda.synchronize()
     t_fill = time.time() - t_fill
     v = pool.views()
@@ -195,8 +209,11 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     attn_events = []
 
+    ids_host = list(ids)
+
     def hot_path(s, time_attn=False):
         pool.append_kv(ids_dev, 1, s["k"], s["v"])
+        append_log.append((ids_host, 1))
         for l in range(L):
             if time_attn:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
@@ -293,7 +310,9 @@ def run_ours(args):
                    "l2_policy": "inputs larger than L2 (%.1f GB of KV per layer call)" % (kv_bytes / 1e9),
                    "multi_gpu": "replicas only (one independent problem per GPU)", "fill_s": round(t_fill, 1)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "traffic": None if ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE is None else algo_bytes * ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE,
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the one-layer 64-trace workload, scaled by algorithmic bytes",
                      "kernel": "decode_attention (attn_mma_kernel + attn_merge_kernel), one layer",
                      "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": attn_avg_ms,
                      "min_launch_ms": float(np.min(attn_ms)), "launches_timed": len(attn_ms)},
@@ -306,6 +325,14 @@ def run_ours(args):
                       "d2h_bytes_per_step": e2e[2], "ms_per_step": e2e[0] * 1e3 / e2e_steps}
     if not args.no_cpu_baseline:
         res["cpu_baseline"], res["sampled_parity"] = cpu_baseline_and_parity(pool, cfg, sets[(K - 1) % NSETS], out, L, phys_layers)
+    if not args.no_aux:
+        res["scorer"] = scorer_measurements(cfg, dev, rows=args.scorer_rows)
+        if args.workload == "c3":
+            # last: this consumes the benchmark state (the pool ends with two live traces)
+            cyc = prune_cycles(pool, cfg, nb, T, dev, wts, append_log, phys_layers, peak)
+            res["prune_cycles"] = cyc["report"]
+            if not args.no_cpu_baseline:
+                res["prune_cycles"]["oracle_replay"] = replay_cycles_on_oracle(cfg, nb, T, max_pages, append_log, cyc["snapshots"])
     print(json.dumps(res))
     if world > 1:
         dist.destroy_process_group()
@@ -361,6 +388,214 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
     return base, par
 
 
+
+# ---------------------------------------------------------------------------------------------
+def scorer_measurements(cfg, dev, rows=65536, reps=20, all_rows_density=1.0):
+    """score_steps timed alone (CUDA events around each call, median of `reps`) on three shapes of one scorer:
+    a decode step (one row per trace, Bernoulli step-end flags), the batched shape (1024 rows per trace at the
+    same density) and `rows` rows that all end a step (scoring every step of many finished traces at once)."""
+    import torch
+    from paper_2601_09093_b200 import binding as B, harness as H, workloads as W
+    T = cfg.n_traces
+    (W1b, _), (b1b, _), (w2b, _), b2 = W.scorer_weights(cfg, bias_std=0.05)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16", dev), H.to_device(b1b, "bf16", dev), H.to_device(w2b, "bf16", dev), b2, B.STEP_BF16)
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 55)
+    shapes = [("decode", T, cfg.boundary_density), ("batched", T * 1024, cfg.boundary_density), ("all_rows", rows, all_rows_density)]
+    Mmax = max(m for _, m, _ in shapes)
+    pool = H.make_pool(W.scaled(cfg, num_layers=1), 8, 4, T, max_score_rows=Mmax, device=dev)
+    hid = torch.randn((Mmax, cfg.scorer_D), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    rt = (torch.arange(Mmax, device=dev) % T).to(torch.int32)
+    out = torch.empty(Mmax, dtype=torch.float32, device=dev)
+    peak, kind = measured_peaks("bf16_tflops", 1590.0)
+    res = {"D": cfg.scorer_D, "m": cfg.scorer_m, "unit": "boundary rows scored per second (scorer calls/s)",
+           "flops_per_row": 2 * cfg.scorer_m * (cfg.scorer_D + 1), "bf16_peak_tflops": peak, "peak_kind": "of " + kind}
+    for name, M, density in shapes:
+        if density >= 1.0:
+            mask = torch.ones(M, dtype=torch.uint8, device=dev)
+        else:
+            mask = torch.from_numpy(W.boundary_mask(cfg, M, sub=900, density=density)).to(dev)
+            if int(mask.sum().item()) == 0:
+                mask[0] = 1
+        for _ in range(3):
+            pool.score_steps(hid[:M], mask, rt[:M], wts, out[:M])
+        info = pool.score_launch_info()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        ev[0].record()
+        for i in range(reps):
+            pool.score_steps(hid[:M], mask, rt[:M], wts, out[:M])
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        ms = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(reps)]))
+        nbr = info["n_rows"]
+        tfl = nbr * res["flops_per_row"] / (ms * 1e-3) / 1e12
+        res[name] = {"rows": M, "boundary_rows": nbr, "us_per_call": ms * 1e3, "rows_per_s": nbr / (ms * 1e-3),
+                     "tflops": tfl, "frac_of_bf16_peak": tfl / peak,
+                     "first_layer": ("tcgen05, %d units per CTA" % info["tc_units"]) if info["tc_units"] else "cuda cores"}
+    code, mask_bits = pool.last_error()
+    res["device_error_mask"] = mask_bits
+    pool.close()
+    return res
+
+
+def prune_cycles(pool, cfg, nb, T, dev, wts, append_log, phys_layers, hbm_peak, n_cycles=5):
+    """The memory-saturated workload proper, continued from the benchmark state: the live traces grow until the
+    pool reaches the trigger (used + need > floor(threshold * total)), every live trace gets a fresh step score,
+    prune_if_saturated keeps the top half and reclaims the rest; five times, 64 -> 2 live traces.  At every
+    saturation point decode_attention of a few layers and the prune call are timed with CUDA events.  Returns the
+    report and, for the oracle's replay, what the GPU decided and left behind at each cycle."""
+    import torch
+    v = pool.views()
+    P, L = cfg.page_size, phys_layers
+    limit = math.floor(float(np.float32(cfg.threshold)) * nb)
+    per_tok = L * cfg.num_kv_heads * cfg.head_dim                       # K (or V) elements of one token
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 77)
+    buf_elems = 1 << 27                                                  # 256 MB of K and of V per append call
+    kbuf = torch.randn(buf_elems, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    vbuf = torch.randn(buf_elems, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    hid = torch.randn((T, cfg.scorer_D), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((T, cfg.num_q_heads, cfg.head_dim), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((T, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
+    step_scores = torch.empty(T, dtype=torch.float32, device=dev)
+    report, snaps = [], []
+    for cyc in range(n_cycles):
+        live_h = torch.nonzero(v["live"][:T]).flatten().cpu().tolist()
+        n_live = len(live_h)
+        if n_live < 2:
+            break
+        live = torch.tensor(live_h, dtype=torch.int32, device=dev)
+        used = pool.stats()["used"]
+        S = int(v["seq_lens"][live_h[0]].item())                         # survivors have equal lengths
+        new_pages = (limit - used) // n_live
+        n_tok = (-(-S // P) + new_pages) * P - S
+        c_max = max(1, buf_elems // (n_live * per_tok))
+        left = n_tok
+        while left > 0:
+            c = min(left, c_max)
+            shape = (n_live, c, L, cfg.num_kv_heads, cfg.head_dim)
+            pool.append_kv(live, c, kbuf[: n_live * c * per_tok].view(shape), vbuf[: n_live * c * per_tok].view(shape))
+            append_log.append((live_h, c))
+            left -= c
+        # decode attention at the saturation point (dead traces have length 0)
+        n_att = 6
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_att + 1)]
+        for l in range(2):
+            pool.decode_attention(l % L, q, v["block_table"], v["seq_lens"], out)
+        ev[0].record()
+        for l in range(n_att):
+            pool.decode_attention((2 + l) % L, q, v["block_table"], v["seq_lens"], out)
+            ev[l + 1].record()
+        torch.cuda.synchronize()
+        att_ms = float(np.mean([ev[i].elapsed_time(ev[i + 1]) for i in range(n_att)]))
+        tokens = S + n_tok
+        kv_bytes = (cfg.prefix_len + n_live * (tokens - cfg.prefix_len)) * cfg.bytes_per_token_layer
+        # a fresh score for every live trace, then the prune
+        mask = v["live"][:T].clone()
+        pool.score_steps(hid, mask, None, wts, step_scores)
+        scores_h = v["trace_scores"].cpu().numpy().copy()
+        st0 = pool.stats()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        pid, npr = pool.prune_if_saturated(None, cfg.threshold, cfg.keep_frac)
+        e1.record()
+        torch.cuda.synchronize()
+        n_pruned = int(npr.item())
+        st1 = pool.stats()
+        fc = int(v["free_count"].item())
+        snaps.append(dict(scores=scores_h, pruned=pid[:n_pruned].cpu().tolist(), free_list=v["free_list"][:fc].cpu().numpy(),
+                          refcount=v["refcount"].cpu().numpy(), seq_lens=v["seq_lens"].cpu().numpy(),
+                          live=v["live"].cpu().numpy(), block_table=v["block_table"].cpu().numpy(), log_pos=len(append_log)))
+        # no waiting queue: every survivor's next token must find a block
+        surv_h = torch.nonzero(v["live"][:T]).flatten().cpu().tolist()
+        surv = torch.tensor(surv_h, dtype=torch.int32, device=dev)
+        shape = (len(surv_h), 1, L, cfg.num_kv_heads, cfg.head_dim)
+        pool.append_kv(surv, 1, kbuf[: len(surv_h) * per_tok].view(shape), vbuf[: len(surv_h) * per_tok].view(shape))
+        append_log.append((surv_h, 1))
+        code, bits = pool.last_error()
+        report.append({"cycle": cyc + 1, "live_before": n_live, "live_after": st1["live_traces"], "tokens_per_trace": tokens,
+                       "used_blocks_before": st0["used"], "blocks_reclaimed": st0["used"] - st1["used"],
+                       "prune_us": e0.elapsed_time(e1) * 1e3, "blocks_reclaimed_per_s": (st0["used"] - st1["used"]) / (e0.elapsed_time(e1) * 1e-3),
+                       "attention_ms_per_layer": att_ms, "attention_kv_gbs": kv_bytes / (att_ms * 1e-3) / 1e9,
+                       "attention_frac_of_hbm_peak": kv_bytes / (att_ms * 1e-3) / 1e9 / hbm_peak,
+                       "survivors_scheduled_next_token": bits == 0, "device_error_mask": bits})
+    return {"report": {"threshold": cfg.threshold, "keep_frac": cfg.keep_frac, "cycles": report}, "snapshots": snaps}
+
+
+def replay_cycles_on_oracle(cfg, nb, T, max_pages, append_log, snaps):
+    """The oracle's pool (bookkeeping only) is taken through the run's every append_kv call and, at each cycle, is
+    given the GPU's trace scores; its evicted set, free list, reference counts, lengths, live flags and block table
+    must equal what the GPU left, bit for bit.  Part of the CPU leg: the oracle's prune is timed too."""
+    from oracle.kv_pool import KVPoolOracle
+    o = KVPoolOracle(cfg.num_layers, cfg.num_kv_heads, cfg.head_dim, cfg.page_size, nb, T, max_pages, store_payload=False)
+    o.fork_prefix(T, cfg.prefix_len)
+    pos, ok, cpu_us, first_bad = 0, True, [], None
+    for k, sn in enumerate(snaps):
+        for ids, n in append_log[pos:sn["log_pos"]]:
+            o.append_kv(ids, n)
+        pos = sn["log_pos"]
+        t0 = time.perf_counter()
+        got = o.prune_if_saturated(sn["scores"], cfg.threshold, cfg.keep_frac)
+        cpu_us.append((time.perf_counter() - t0) * 1e6)
+        same = (got == sn["pruned"] and o.free_list == sn["free_list"].tolist()
+                and np.array_equal(o.refcount, sn["refcount"]) and np.array_equal(o.seq_lens, sn["seq_lens"])
+                and np.array_equal(o.live, sn["live"].astype(bool)) and np.array_equal(o.block_table, sn["block_table"]))
+        if not same and first_bad is None:
+            first_bad = k + 1
+        ok = ok and same
+    return {"what": "evicted ids, free list, refcounts, lengths, live flags and block table after each prune, bit-exact "
+                    "against the oracle replaying all %d append_kv calls with the GPU's scores" % len(append_log),
+            "ok": bool(ok), "first_mismatching_cycle": first_bad, "oracle_prune_us": cpu_us, "status_bits": int(o.status)}
+
+
+# ---------------------------------------------------------------------------------------------
+def run_scorer(args):
+    """`--workload scorer`: score_steps alone on a large batch of step-end hidden states (every step of many
+    finished traces scored at once).  The line's roofline is the tensor-core one of the first-layer GEMM."""
+    import torch
+    from paper_2601_09093_b200 import binding as B, workloads as W
+    from paper_2601_09093_b200 import build as _build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        _build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    B.lib()
+    cfg = {"c1": W.C1, "c4": W.C4}[args.scorer_shape]
+    K = max(args.steps, 3)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    m = scorer_measurements(cfg, dev, rows=args.scorer_rows, reps=K, all_rows_density=args.scorer_density)
+    clocks = sampler.stop() if rank == 0 else None
+    a = m["all_rows"]
+    if world > 1:
+        tt = torch.tensor([a["us_per_call"]], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        a["us_per_call"] = float(tt[0]); a["rows_per_s"] = a["boundary_rows"] / (a["us_per_call"] * 1e-6)
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    flops = a["boundary_rows"] * m["flops_per_row"]
+    res = {"metric": "scorer calls/s (step-end hidden states scored per second)", "value": world * a["rows_per_s"],
+           "unit": "rows/s", "n_gpus": world, "steps": K, "warmup": 3, "ms_per_step": a["us_per_call"] * 1e-3,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic (seeded, drawn on device)",
+           "config": {"workload": "scorer-batched-%s" % cfg.name, "rows": a["rows"], "boundary_rows": a["boundary_rows"],
+                      "D": cfg.scorer_D, "m": cfg.scorer_m, "first_layer": a["first_layer"],
+                      "l2_policy": "inputs larger than L2 (%.0f MB of hidden states per call)" % (a["rows"] * cfg.scorer_D * 2 / 1e6)},
+           "roofline": {"bound": "tensor", "achieved": a["tflops"], "peak": m["bf16_peak_tflops"], "unit": "TFLOP/s",
+                        "frac": a["frac_of_bf16_peak"], "peak_kind": m["peak_kind"] + " (burst: the call is timed alone)",
+                        "traffic": None, "kernel": "score_steps (compact + score_tc_kernel + finish), whole call",
+                        "algorithmic_flops_per_launch": flops},
+           "scorer": m, "gpu_launches": 3 * K, "clocks": clocks}
+    print(json.dumps(res))
+
+
 # ---------------------------------------------------------------------------------------------
 def run_reference(args):
     """The reference arm of this build is the CPU oracle, as it stands, on the host cores."""
@@ -372,6 +607,8 @@ def run_reference(args):
     from paper_2601_09093_b200 import workloads as W
 
     K, Wm = args.steps, max(args.warmup, 1)
+    if args.workload == "scorer":
+        return run_reference_scorer(args, K, Wm)
     cfg, suffix, nb, max_pages, _ = workload_plan(args.workload, args.num_blocks, Wm + K + 4)
     T, L, P = cfg.n_traces, cfg.num_layers, cfg.page_size
     # bounded sample of one step: attention of ONE trace in ONE layer at the benchmark's length,
@@ -423,9 +660,42 @@ def run_reference(args):
     print(json.dumps(res))
 
 
+def run_reference_scorer(args, K, Wm, sample=64):
+    """The oracle's scorer on a bounded sample (64 step-end rows per step) of the batched scorer workload."""
+    from oracle import scorer as OS
+    from paper_2601_09093_b200 import workloads as W
+    cfg = {"c1": W.C1, "c4": W.C4}[args.scorer_shape]
+    (_, W1x), (_, b1x), (_, w2x), b2 = W.scorer_weights(cfg, bias_std=0.05)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    mask = np.ones(sample, dtype=np.uint8)
+
+    def step(i):
+        _, hx = W.normal(cfg.seed, W.TID_HID, (sample, cfg.scorer_D), "bf16", sub=i)
+        OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+
+    for i in range(Wm):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(K):
+        step(Wm + i)
+    dt = time.perf_counter() - t0
+    value = K * sample / dt
+    unit = "rows/s"
+    print(json.dumps({"impl": "reference", "metric": "scorer calls/s (step-end hidden states scored per second)", "value": value,
+                      "unit": unit, "n_gpus": args.gpus, "steps": K, "warmup": Wm, "ms_per_step": dt * 1e3 / K,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+                      "config": {"workload": "scorer-batched-%s" % cfg.name, "D": cfg.scorer_D, "m": cfg.scorer_m,
+                                 "note": "CPU oracle; each step scores %d rows" % sample},
+                      "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle",
+                                       "sample": "%d step-end rows per step" % sample},
+                      "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.workload == "scorer":
+        run_scorer(a)
     else:
         run_ours(a)

@@ -45,12 +45,13 @@ def ragged_append_plan(lengths):
             done += inc
 
 
-def fill_random_device(pool: B.KVPool, cfg: W.Config, lengths, seed: int, chunk_tokens=2048):
+def fill_random_device(pool: B.KVPool, cfg: W.Config, lengths, seed: int, chunk_tokens=2048, log=None):
     """Forks cfg.n_traces traces from a random prompt and grows trace i by lengths[i] tokens.
 
     K/V values are N(0,1) drawn ON THE DEVICE from a seeded torch generator (the pools of the large
     configurations are far too big to draw on the host); parity tests read the stored rows back
-    through kv_pool_read_kv and hand those bytes to the oracle.
+    through kv_pool_read_kv and hand those bytes to the oracle.  `log`, if given, receives one
+    (trace id list, n_tokens) entry per append_kv call, in call order.
     """
     dev = pool.device
     gen = torch.Generator(device=dev)
@@ -69,6 +70,8 @@ def fill_random_device(pool: B.KVPool, cfg: W.Config, lengths, seed: int, chunk_
             kn = torch.randn((len(sel), c, L, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(tdt)
             vn = torch.randn((len(sel), c, L, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(tdt)
             pool.append_kv(tid, c, kn, vn)
+            if log is not None:
+                log.append((ids_np[sel].tolist(), c))
             left -= c
     return ids
 
