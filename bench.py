@@ -149,12 +149,10 @@ def workload_plan(name, num_blocks_override, steps_total, free_bytes=None):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2601_09093_b200 import binding as B, harness as H, workloads as W
+    from paper_2601_09093_b200 import binding as B, harness as H, ranks as R, workloads as W
     from paper_2601_09093_b200 import build as _build
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = R.rank_env()
     if rank == 0:
         _build.build()
     torch.cuda.set_device(local_rank)
@@ -276,15 +274,9 @@ def run_ours(args):
         d2h = host_out.numel() * 4 + host_scores.numel() * 4 + host_tscores.numel() * 4 + 4
         e2e = (e2e_s, h2d, d2h)
 
-    if world > 1:
-        tt = torch.tensor([ms_total, e2e[0] if e2e else 0.0], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt[0]); e2e = (float(tt[1]), e2e[1], e2e[2]) if e2e else None
-        ok = torch.tensor([int(err_mask == 0 and n_live == T)], device=dev)
-        dist.all_reduce(ok, op=dist.ReduceOp.MIN)
-        all_ok = bool(ok.item())
-    else:
-        all_ok = err_mask == 0 and n_live == T
+    (ms_total, e2e_max), all_ok = R.max_over_ranks([ms_total, e2e[0] if e2e else 0.0], err_mask == 0 and n_live == T, dev)
+    if e2e:
+        e2e = (e2e_max, e2e[1], e2e[2])
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -298,7 +290,7 @@ def run_ours(args):
     algo_bytes = kv_bytes + T * cfg.num_q_heads * cfg.head_dim * (2 + 4) + pages * 4
     attn_avg_ms = float(np.mean(attn_ms))
     achieved = algo_bytes / (attn_avg_ms * 1e-3) / 1e9
-    value = world * T * K / (ms_total * 1e-3)
+    value = R.whole_job_rate(T * K, world, ms_total * 1e-3)
     res = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -321,7 +313,7 @@ def run_ours(args):
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
     if e2e:
-        res["e2e"] = {"value": world * T * e2e_steps / e2e[0], "unit": UNIT, "h2d_bytes_per_step": e2e[1],
+        res["e2e"] = {"value": R.whole_job_rate(T * e2e_steps, world, e2e[0]), "unit": UNIT, "h2d_bytes_per_step": e2e[1],
                       "d2h_bytes_per_step": e2e[2], "ms_per_step": e2e[0] * 1e3 / e2e_steps}
     if not args.no_cpu_baseline:
         res["cpu_baseline"], res["sampled_parity"] = cpu_baseline_and_parity(pool, cfg, sets[(K - 1) % NSETS], out, L, phys_layers)
@@ -551,11 +543,9 @@ def run_scorer(args):
     """`--workload scorer`: score_steps alone on a large batch of step-end hidden states (every step of many
     finished traces scored at once).  The line's roofline is the tensor-core one of the first-layer GEMM."""
     import torch
-    from paper_2601_09093_b200 import binding as B, workloads as W
+    from paper_2601_09093_b200 import binding as B, ranks as R, workloads as W
     from paper_2601_09093_b200 import build as _build
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = R.rank_env()
     if rank == 0:
         _build.build()
     torch.cuda.set_device(local_rank)
@@ -573,15 +563,14 @@ def run_scorer(args):
     m = scorer_measurements(cfg, dev, rows=args.scorer_rows, reps=K, all_rows_density=args.scorer_density)
     clocks = sampler.stop() if rank == 0 else None
     a = m["all_rows"]
+    (a["us_per_call"],), _ = R.max_over_ranks([a["us_per_call"]], m["device_error_mask"] == 0, dev)
+    a["rows_per_s"] = a["boundary_rows"] / (a["us_per_call"] * 1e-6)
     if world > 1:
-        tt = torch.tensor([a["us_per_call"]], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        a["us_per_call"] = float(tt[0]); a["rows_per_s"] = a["boundary_rows"] / (a["us_per_call"] * 1e-6)
         dist.destroy_process_group()
     if rank != 0:
         return
     flops = a["boundary_rows"] * m["flops_per_row"]
-    res = {"metric": "scorer calls/s (step-end hidden states scored per second)", "value": world * a["rows_per_s"],
+    res = {"metric": "scorer calls/s (step-end hidden states scored per second)", "value": R.whole_job_rate(a["boundary_rows"], world, a["us_per_call"] * 1e-6),
            "unit": "rows/s", "n_gpus": world, "steps": K, "warmup": 3, "ms_per_step": a["us_per_call"] * 1e-3,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
            "data": "synthetic (seeded, drawn on device)",
@@ -598,9 +587,10 @@ def run_scorer(args):
 
 # ---------------------------------------------------------------------------------------------
 def run_reference(args):
-    """The reference arm of this build is the CPU oracle, as it stands, on the host cores."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """The reference arm of this build is the CPU oracle, as it stands, on the host cores.
+    Under a multi-rank launcher rank 0 alone runs and prints; the other ranks leave at once."""
+    from paper_2601_09093_b200 import ranks as R
+    if R.rank_env()[0] != 0:
         return
     from oracle import attention as OA, scorer as OS
     from oracle.kv_pool import KVPoolOracle
