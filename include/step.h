@@ -157,6 +157,27 @@ int score_steps(step_pool* pool, const void* hidden, const uint8_t* boundary_mas
                 const int32_t* row_trace, int M, const scorer_weights* weights,
                 float* step_scores_out, void* stream);
 
+/* Step-end detection (Sec. 3.1 "Step Representation" and its footnote; Algorithm 1: `if "\n\n" in x`):
+ * a sampled token ends a reasoning step if its text contains two consecutive newline characters.
+ * step_end_table_from_vocab fills table_out[v] (HOST, vocab bytes) with 1 for such vocabulary entries and 0
+ * for the others; token_text[v] (HOST) is the entry's text, text_len[v] its length in bytes, or text_len =
+ * NULL for NUL-terminated strings; a NULL entry counts as empty.  Needs no GPU. */
+int step_end_table_from_vocab(const char* const* token_text, const int32_t* text_len, int vocab,
+                              uint8_t* table_out);
+/* boundary_mask_out[i] = step_end_table[token_ids[i]] for M sampled tokens (device pointers; the table is a
+ * device copy of what step_end_table_from_vocab made).  An id outside [0, vocab) ends no step and sets the
+ * STEP_ERR_INVALID_ARG bit of the device status word. */
+int detect_step_ends(step_pool* pool, const int32_t* token_ids, int M, const uint8_t* step_end_table,
+                     int vocab, uint8_t* boundary_mask_out, void* stream);
+/* score_steps with the step-end flags taken from the sampled tokens instead of a mask: row i is scored iff
+ * step_end_table[token_ids[i]] != 0 (one pass less over the rows than detect_step_ends + score_steps).
+ * The flags are also written to boundary_mask_out (device, [M]) unless it is NULL.  Everything else as
+ * score_steps. */
+int score_steps_tokens(step_pool* pool, const void* hidden, const int32_t* token_ids,
+                       const uint8_t* step_end_table, int vocab, const int32_t* row_trace, int M,
+                       const scorer_weights* weights, float* step_scores_out, uint8_t* boundary_mask_out,
+                       void* stream);
+
 /* Memory trigger and eviction (Sec. 3.2, Algorithm 1):
  *   used = total - free_count; need = #{live t: S_t % page_size == 0};
  *   saturated <=> used + need > floor((double)threshold * total).

@@ -64,6 +64,9 @@ def lib():
     L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_static.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
+    L.score_steps_tokens.argtypes = [vp, vp, vp, vp, i, vp, i, C.POINTER(scorer_weights), vp, vp, vp]
+    L.detect_step_ends.argtypes = [vp, vp, i, vp, i, vp, vp]
+    L.step_end_table_from_vocab.argtypes = [C.POINTER(C.c_char_p), ip, i, vp]
     L.prune_if_saturated.argtypes = [vp, vp, C.c_float, C.c_float, vp, vp, vp]
     L.kv_pool_release_traces.argtypes = [vp, vp, i, vp]
     L.kv_pool_stats.argtypes = [vp, ip, ip, ip, ip, vp]
@@ -198,6 +201,24 @@ class KVPool:
                                                 C.byref(weights.struct), _ptr(step_scores_out), _stream(stream)))
         return step_scores_out
 
+    def score_steps_tokens(self, hidden, token_ids, step_end_table, row_trace, weights, step_scores_out=None,
+                           boundary_mask_out=None, stream=None):
+        M = hidden.shape[0]
+        if step_scores_out is None:
+            step_scores_out = torch.empty(M, dtype=torch.float32, device=hidden.device)
+        _check("score_steps_tokens", lib().score_steps_tokens(
+            self.handle, _ptr(hidden), _ptr(token_ids), _ptr(step_end_table), step_end_table.numel(), _ptr(row_trace), M,
+            C.byref(weights.struct), _ptr(step_scores_out), _ptr(boundary_mask_out), _stream(stream)))
+        return step_scores_out
+
+    def detect_step_ends(self, token_ids, step_end_table, boundary_mask_out=None, stream=None):
+        M = token_ids.numel()
+        if boundary_mask_out is None:
+            boundary_mask_out = torch.empty(M, dtype=torch.uint8, device=token_ids.device)
+        _check("detect_step_ends", lib().detect_step_ends(self.handle, _ptr(token_ids), M, _ptr(step_end_table),
+                                                          step_end_table.numel(), _ptr(boundary_mask_out), _stream(stream)))
+        return boundary_mask_out
+
     def prune_if_saturated(self, scores, threshold, keep_frac, stream=None):
         """Returns (pruned_ids, n_pruned) device tensors owned by the pool (no sync)."""
         _check("prune_if_saturated", lib().prune_if_saturated(self.handle, _ptr(scores), threshold, keep_frac,
@@ -235,6 +256,17 @@ class KVPool:
         n, u = C.c_int(), C.c_int()
         _check("kv_pool_score_launch_info", lib().kv_pool_score_launch_info(self.handle, C.byref(n), C.byref(u), _stream(stream)))
         return dict(n_rows=n.value, tc_units=u.value)
+
+
+def step_end_table_from_vocab(token_texts):
+    """Host table (torch.uint8, [vocab]) marking the vocabulary entries whose text contains two newlines in a row.
+    token_texts: a sequence of bytes objects (None = empty)."""
+    n = len(token_texts)
+    arr = (C.c_char_p * n)(*[t if t is not None else None for t in token_texts])
+    lens = (C.c_int * n)(*[len(t) if t is not None else 0 for t in token_texts])
+    out = torch.zeros(n, dtype=torch.uint8)
+    _check("step_end_table_from_vocab", lib().step_end_table_from_vocab(arr, lens, n, C.c_void_p(out.data_ptr())))
+    return out
 
 
 class ScorerWeights:

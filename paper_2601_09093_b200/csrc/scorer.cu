@@ -35,10 +35,32 @@ template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return
 // tc_min_rows: 0 = the tensor-core kernel is not available for this launch; otherwise the smallest
 // number of boundary rows that goes to it.  m: hidden units; num_sms: for the tiling choice.
 // One CTA; a thread looks at kRowsPerThread consecutive rows per pass.
+// The step-end flag of row i is either mask[i] (tokens == nullptr) or, when the caller hands over the
+// sampled token ids instead, table[tokens[i]]: a token ends a step if its text contains "\n\n" (Sec. 3.1,
+// footnote), which the table records per vocabulary entry.  In that case the flags are also written to
+// mask_out if it is given.  An id outside the vocabulary ends no step and is flagged.
 constexpr int kRowsPerThread = 8;
 
+struct FlagSource {
+  const uint8_t* mask;       // [M], or nullptr
+  const int32_t* tokens;     // [M], or nullptr
+  const uint8_t* table;      // [vocab]
+  int vocab;
+  uint8_t* mask_out;         // [M], or nullptr
+};
+
+__device__ inline bool row_flag(const FlagSource& f, int i, int32_t* counters) {
+  if (!f.tokens) return f.mask[i] != 0;
+  const int id = f.tokens[i];
+  bool e = false;
+  if (id < 0 || id >= f.vocab) flag_error(counters, STEP_ERR_INVALID_ARG);
+  else e = f.table[id] != 0;
+  if (f.mask_out) f.mask_out[i] = e ? 1 : 0;
+  return e;
+}
+
 __global__ void __launch_bounds__(kCompactThreads)
-score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float* __restrict__ step_scores,
+score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step_scores,
                      int tc_min_rows, int m, int num_sms) {
   __shared__ int s_warp[33];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -49,7 +71,7 @@ score_compact_kernel(DevViews v, const uint8_t* __restrict__ mask, int M, float*
     unsigned flags = 0;
 #pragma unroll
     for (int j = 0; j < kRowsPerThread; ++j)
-      if (i0 + j < M && mask[i0 + j] != 0) flags |= 1u << j;
+      if (i0 + j < M && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
     const int mine = __popc(flags);
     int incl = mine;
 #pragma unroll
@@ -214,6 +236,15 @@ score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, in
   }
 }
 
+// step-end detection alone: mask[i] = table[tokens[i]]
+__global__ void __launch_bounds__(256)
+step_end_kernel(FlagSource src, int M, int32_t* counters) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < M; i += gridDim.x * blockDim.x) row_flag(src, i, counters);
+}
+
+int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
+                     const scorer_weights* w, float* step_scores_out, void* stream);
+
 }  // namespace
 
 extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* boundary_mask,
@@ -221,7 +252,59 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
                            float* step_scores_out, void* stream) {
   if (!pool || M < 0 || !w) return STEP_ERR_INVALID_ARG;
   if (M == 0) return STEP_OK;
-  if (!hidden || !boundary_mask || !step_scores_out) return STEP_ERR_INVALID_ARG;
+  if (!boundary_mask) return STEP_ERR_INVALID_ARG;
+  FlagSource src{boundary_mask, nullptr, nullptr, 0, nullptr};
+  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
+}
+
+extern "C" int score_steps_tokens(step_pool* pool, const void* hidden, const int32_t* token_ids,
+                                  const uint8_t* step_end_table, int vocab, const int32_t* row_trace, int M,
+                                  const scorer_weights* w, float* step_scores_out, uint8_t* boundary_mask_out,
+                                  void* stream) {
+  if (!pool || M < 0 || !w) return STEP_ERR_INVALID_ARG;
+  if (M == 0) return STEP_OK;
+  if (!token_ids || !step_end_table || vocab < 1) return STEP_ERR_INVALID_ARG;
+  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out};
+  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
+}
+
+extern "C" int detect_step_ends(step_pool* pool, const int32_t* token_ids, int M, const uint8_t* step_end_table,
+                                int vocab, uint8_t* boundary_mask_out, void* stream) {
+  if (!pool || M < 0) return STEP_ERR_INVALID_ARG;
+  if (M == 0) return STEP_OK;
+  if (!token_ids || !step_end_table || vocab < 1 || !boundary_mask_out) return STEP_ERR_INVALID_ARG;
+  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out};
+  int ctas = (M + 255) / 256;
+  if (ctas > pool->num_sms * 8) ctas = pool->num_sms * 8;
+  step_end_kernel<<<ctas, 256, 0, (cudaStream_t)stream>>>(src, M, pool->v.counters);
+  return launch_ok();
+}
+
+extern "C" int step_end_table_from_vocab(const char* const* token_text, const int32_t* text_len, int vocab,
+                                         uint8_t* table_out) {
+  if (!token_text || vocab < 0 || !table_out) return STEP_ERR_INVALID_ARG;
+  for (int v = 0; v < vocab; ++v) {
+    const char* t = token_text[v];
+    uint8_t hit = 0;
+    if (t) {
+      if (text_len) {
+        for (int i = 0; i + 1 < text_len[v]; ++i)
+          if (t[i] == '\n' && t[i + 1] == '\n') { hit = 1; break; }
+      } else {
+        for (int i = 0; t[i] && t[i + 1]; ++i)
+          if (t[i] == '\n' && t[i + 1] == '\n') { hit = 1; break; }
+      }
+    }
+    table_out[v] = hit;
+  }
+  return STEP_OK;
+}
+
+namespace {
+
+int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
+                     const scorer_weights* w, float* step_scores_out, void* stream) {
+  if (!hidden || !step_scores_out) return STEP_ERR_INVALID_ARG;
   if (!w->W1 || !w->b1 || !w->w2 || w->D < 1 || w->m < 1) return STEP_ERR_INVALID_ARG;
   if (w->dtype != STEP_BF16 && w->dtype != STEP_FP32) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)kRowTile * w->D * sizeof(float);
@@ -235,7 +318,11 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
     const int Mc = M - off < pool->max_score_rows ? M - off : pool->max_score_rows;
     const char* hid = (const char*)hidden + (size_t)off * w->D * eb;
     const int32_t* rt = row_trace ? row_trace + off : nullptr;
-    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, boundary_mask + off, Mc, step_scores_out + off,
+    FlagSource part = src;
+    if (part.mask) part.mask += off;
+    if (part.tokens) part.tokens += off;
+    if (part.mask_out) part.mask_out += off;
+    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, part, Mc, step_scores_out + off,
                                                        tc_min_rows, w->m, pool->num_sms);
     // the CUDA-core kernel only ever sees launches with fewer than tc_min_rows boundary rows
     const int scalar_rows = tc_min_rows > 0 && tc_min_rows - 1 < Mc ? tc_min_rows - 1 : Mc;
@@ -263,6 +350,8 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
   }
   return launch_ok();
 }
+
+}  // namespace
 
 extern "C" int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows) {
   if (!pool || mode < -1 || mode > 1 || tc_min_rows < 0) return STEP_ERR_INVALID_ARG;

@@ -25,7 +25,7 @@ import numpy as np
 
 # tensor ids (second half of the Philox key)
 TID_Q, TID_K, TID_V, TID_KPRE, TID_VPRE, TID_LEN, TID_HID, TID_MASK = 1, 2, 3, 4, 5, 6, 7, 8
-TID_W1, TID_W2, TID_B1, TID_PERM, TID_ANS, TID_KNEW, TID_VNEW = 9, 10, 11, 12, 13, 14, 15
+TID_W1, TID_W2, TID_B1, TID_PERM, TID_ANS, TID_KNEW, TID_VNEW, TID_VOCAB, TID_TOK = 9, 10, 11, 12, 13, 14, 15, 16, 17
 
 
 @dataclasses.dataclass(frozen=True)
@@ -155,3 +155,32 @@ def block_permutation(seed: int, num_blocks: int) -> np.ndarray:
 def scaled(cfg: Config, **kw) -> Config:
     """A copy of cfg with some fields replaced (cut-down variants for tests)."""
     return dataclasses.replace(cfg, **kw)
+
+
+def synthetic_vocab(seed: int, vocab_size: int, step_end_frac: float = 0.01):
+    """A stand-in for a tokenizer's vocabulary: `vocab_size` byte strings of 1-8 bytes drawn from letters, digits,
+    space, punctuation and the newline character; about `step_end_frac` of the entries get two newlines in a row
+    planted somewhere (entries may also contain them by chance, or single and separated newlines, which do not
+    count).  Entry 0 is empty.  Returns a list of bytes."""
+    g = rng(seed, TID_VOCAB)
+    alphabet = np.frombuffer(b"abcdefghijklmnopqrstuvwxyzABCDEFGHIJKLMNOPQRSTUVWXYZ0123456789 .,:;()=+-\n", dtype=np.uint8)
+    out = [b""]
+    for v in range(1, vocab_size):
+        n = int(g.integers(1, 9))
+        t = bytearray(alphabet[g.integers(0, len(alphabet), size=n)].tobytes())
+        if g.random() < step_end_frac:
+            at = int(g.integers(0, n + 1))
+            t[at:at] = b"\n\n"
+        out.append(bytes(t))
+    return out
+
+
+def token_ids(seed: int, n_rows: int, vocab_size: int, step_end_ids, density: float, sub: int = 0) -> np.ndarray:
+    """Sampled-token stand-ins: row i is one of `step_end_ids` with probability `density`, else a uniformly drawn id
+    (which may itself end a step).  int32."""
+    g = rng(seed, TID_TOK, sub)
+    ids = g.integers(0, vocab_size, size=n_rows).astype(np.int32)
+    if len(step_end_ids) and density > 0:
+        pick = g.random(n_rows) < density
+        ids[pick] = np.asarray(step_end_ids, dtype=np.int32)[g.integers(0, len(step_end_ids), size=int(pick.sum()))]
+    return ids

@@ -335,3 +335,55 @@ def test_scorer_running_mean_accumulates_across_calls():
     ts = OS.TraceScores(64)
     ts.update(g1, m1); ts.update(g2, mask)
     np.testing.assert_allclose(pool.views()["trace_scores"].cpu().numpy(), ts.scores(), atol=1e-6)
+
+
+# ------------------------------------------------------------------ step-end detection from sampled tokens
+def _vocab_case(seed, vocab_size, M, density):
+    from oracle import steps as OSt
+    vocab = W.synthetic_vocab(seed, vocab_size, step_end_frac=0.02)
+    table = B.step_end_table_from_vocab(vocab)
+    ends = np.flatnonzero(table.numpy())
+    ids = W.token_ids(seed, M, vocab_size, ends, density)
+    return vocab, table.cuda(), ids, OSt.step_end_mask(ids, vocab)
+
+
+def test_detect_step_ends_matches_the_oracle_bit_for_bit():
+    pool = H.make_pool(W.C0, 8, 4, 8)
+    for M in (1, 255, 4097, 70001):
+        vocab, table, ids, want = _vocab_case(5, 32000, M, 1.0 / 64)
+        got = pool.detect_step_ends(torch.from_numpy(ids).cuda(), table).cpu().numpy()
+        np.testing.assert_array_equal(got, want)
+    assert pool.last_error() == (0, 0)
+    ids[3], ids[9] = -7, 32000                                   # ids outside the vocabulary end no step, and are flagged
+    got = pool.detect_step_ends(torch.from_numpy(ids).cuda(), table).cpu().numpy()
+    assert got[3] == 0 and got[9] == 0
+    assert pool.last_error()[1] == 1 << 1
+
+
+@pytest.mark.parametrize("mode", [-1, 0])
+def test_score_steps_tokens_equals_score_steps_on_the_oracle_mask(mode):
+    cfg = W.C1
+    M = 64 * 30 + 5
+    vocab, table, ids, mask = _vocab_case(cfg.seed, 32000, M, 1.0 / 16)
+    rt = (np.arange(M) % 64).astype(np.int32)
+    pool_a, wts, g_mask, _ = _scorer_case(cfg, M, 0.0, row_trace=rt, max_score_rows=1000, mode=mode)   # builds pool + weights
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (M, cfg.scorer_D), cfg.dtype)
+    hid = H.to_device(hb, cfg.dtype)
+    rt_dev = torch.from_numpy(rt).cuda()
+    ref = pool_a.score_steps(hid, torch.from_numpy(mask).cuda(), rt_dev, wts).cpu().numpy()
+    ref_scores = pool_a.views()["trace_scores"].cpu().numpy().copy()
+    pool_b = H.make_pool(cfg, 8, 4, 64, max_score_rows=1000)
+    pool_b.set_scorer_config(mode, 0)
+    mask_out = torch.empty(M, dtype=torch.uint8, device="cuda")
+    got = pool_b.score_steps_tokens(hid, torch.from_numpy(ids).cuda(), table, rt_dev, wts, boundary_mask_out=mask_out).cpu().numpy()
+    np.testing.assert_array_equal(mask_out.cpu().numpy(), mask)
+    np.testing.assert_array_equal(got, ref)                     # same kernels, same rows: identical bits (NaN where no step ends)
+    np.testing.assert_array_equal(pool_b.views()["trace_scores"].cpu().numpy(), ref_scores)
+    want = OS.score_steps(hx, mask, *[x for x in _exact_weights(cfg)])
+    assert np.abs(got[mask == 1] - want[mask == 1]).max() <= SCORE_TOL
+    assert pool_b.last_error() == (0, 0)
+
+
+def _exact_weights(cfg):
+    (_, W1x), (_, b1x), (_, w2x), b2 = W.scorer_weights(cfg, bias_std=0.05)
+    return W1x, b1x, w2x, b2
