@@ -1,121 +1,31 @@
 // prune_if_saturated: memory trigger, ranking and KV release (Sec. 3.2; Algorithm 1, the
 // GPUMemoryFull branch: t* = argmin score_t, ReleaseKVCache(t*), T <- T \ {t*}).
 //
-// One CTA does the whole call (the trace set is tiny; the block-id traffic is a few hundred KB):
-//   1. predicate   used + need > floor(threshold * total)
+// One thread-block cluster of eight CTAs does the whole call:
+//   1. predicate   used + need > floor(threshold * total)              (every CTA; all leave if it is false)
 //   2. rank        every live trace counts the live traces that order before it
 //                  (score descending, id ascending, NaN last) - a warp per trace, lanes over rivals
-//   3. list        evicted ids in ascending order by a block-wide prefix sum
+//   3. list        evicted ids in ascending order by a block-wide prefix sum          (2, 3: the leading CTA)
 //   4. release     all (trace, page) entries drop one reference in parallel; the entry that is the
 //                  LAST in (trace, page) order to name a block whose count reached zero owns the
-//                  push, and a block-wide prefix sum over the entries in order gives each push its
-//                  place - so the free list comes out exactly as a serial walk would leave it.
-#include "step_internal.cuh"
-
-#include <math.h>
+//                  push; prefix sums within each CTA and push counts exchanged through distributed shared
+//                  memory give each push its place - so the free list comes out exactly as a serial walk
+//                  would leave it.  The entries are spread over the cluster's eight SMs because a release is
+//                  bound by how many scattered 4-byte requests one SM can issue.
+#include "release.cuh"
 
 using namespace stepk;
 
 namespace {
 
-constexpr int kPruneThreads = 1024;
-
-// Exclusive prefix sum of one int per thread over the CTA; *total gets the sum.
-__device__ inline int block_excl_scan(int x, int* s_warp, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = x;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  __syncthreads();                       // s_warp may still be read from the previous call
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    int w = s_warp[lane];
-    int wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += v;
-    }
-    s_warp[lane] = wi - w;               // exclusive offset of each warp
-    if (lane == 31) s_warp[32] = wi;
-  }
-  __syncthreads();
-  *total = s_warp[32];
-  return s_warp[warp] + incl - x;
-}
-
-// true if trace a orders strictly before trace b (a is the better one)
-__device__ inline bool orders_before(float sa, int a, float sb, int b) {
-  const bool na = isnan(sa), nb = isnan(sb);
-  if (na != nb) return nb;               // a number beats NaN
-  if (!na && sa != sb) return sa > sb;
-  return a < b;
-}
-
-// Releases the traces listed in v.prune_list[0 .. n_list) (processed in list order).
-__device__ void release_listed(DevViews& v, const Geo& g, int n_list, float unscored, int* s_warp) {
-  // offsets of each trace's entries in the global (trace, page) order
-  if (threadIdx.x == 0) {
-    int off = 0;
-    for (int k = 0; k < n_list; ++k) {
-      v.prune_off[k] = off;
-      const int S = v.seq_lens[v.prune_list[k]];
-      off += (S + g.P - 1) / g.P;
-    }
-    v.prune_off[n_list] = off;
-  }
-  __syncthreads();
-  // pass A: drop references, find the last entry naming each block
-  for (int k = 0; k < n_list; ++k) {
-    const int t = v.prune_list[k], off = v.prune_off[k], np = v.prune_off[k + 1] - off;
-    const int32_t* row = v.block_table + (size_t)t * g.max_pages;
-    for (int p = threadIdx.x; p < np; p += blockDim.x) {
-      const int b = row[p];
-      if (b < 0 || b >= g.num_blocks) { flag_error(v.counters, STEP_ERR_BAD_BLOCK); continue; }
-      atomicSub(&v.refcount[b], 1);
-      atomicMax(&v.claim[b], off + p);
-    }
-  }
-  __syncthreads();
-  // pass B: pushes in (trace, page) order
-  const int fc = v.counters[C_FREE_COUNT];
-  int pushed = 0;
-  for (int k = 0; k < n_list; ++k) {
-    const int t = v.prune_list[k], off = v.prune_off[k], np = v.prune_off[k + 1] - off;
-    int32_t* row = v.block_table + (size_t)t * g.max_pages;
-    for (int base = 0; base < np; base += blockDim.x) {
-      const int p = base + threadIdx.x;
-      int b = -1, f = 0;
-      if (p < np) {
-        b = row[p];
-        row[p] = -1;
-        if (b >= 0 && b < g.num_blocks && v.claim[b] == off + p) {
-          v.claim[b] = -1;
-          f = v.refcount[b] == 0;
-        }
-      }
-      int chunk_total;
-      const int at = block_excl_scan(f, s_warp, &chunk_total);
-      if (f) v.free_list[fc + pushed + at] = b;
-      pushed += chunk_total;
-    }
-  }
-  for (int k = threadIdx.x; k < n_list; k += blockDim.x) {
-    const int t = v.prune_list[k];
-    v.seq_lens[t] = 0; v.live[t] = 0;
-    v.score_sum[t] = 0.f; v.score_cnt[t] = 0; v.trace_scores[t] = unscored;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) v.counters[C_FREE_COUNT] = fc + pushed;
-}
-
-__global__ void __launch_bounds__(kPruneThreads)
+// A cluster of kClusterCtas CTAs.  Every CTA evaluates the trigger (same inputs, same answer); rank 0 ranks the
+// traces and lists the evicted ones; the cluster releases them together.
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kPruneThreads, 1)
 prune_kernel(DevViews v, Geo g, const float* __restrict__ scores_in, float threshold, float keep_frac,
              float unscored, int32_t* __restrict__ pruned_ids_out, int32_t* __restrict__ n_pruned_out) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const bool leader = cluster.block_rank() == 0;
   __shared__ int s_warp[33];
   __shared__ int s_nlive, s_need, s_go, s_nkeep;
   const float* scores = scores_in ? scores_in : v.trace_scores;
@@ -140,59 +50,64 @@ prune_kernel(DevViews v, Geo g, const float* __restrict__ scores_in, float thres
       if (s_nlive == 0 || n_keep >= s_nlive) go = 0;
     }
     s_go = go; s_nkeep = n_keep;
-    if (!go) *n_pruned_out = 0;
+    if (!go && leader) *n_pruned_out = 0;
   }
   __syncthreads();
-  if (!s_go) return;
+  if (!s_go) return;                      // the whole cluster leaves: nothing has been written yet
   const int n_keep = s_nkeep;
-  // ---- 2. rank by counting: a warp per trace, lanes over rivals
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  for (int t = warp; t < T; t += nwarps) {
-    int evict = 0;
-    if (v.live[t]) {
-      const float st = scores[t];
-      int ahead = 0;
-      for (int u = lane; u < T; u += 32)
-        if (u != t && v.live[u] && orders_before(scores[u], u, st, t)) ++ahead;
+  if (leader) {
+    // ---- 2. rank by counting: a warp per trace, lanes over rivals
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int t = warp; t < T; t += nwarps) {
+      int evict = 0;
+      if (v.live[t]) {
+        const float st = scores[t];
+        int ahead = 0;
+        for (int u = lane; u < T; u += 32)
+          if (u != t && v.live[u] && orders_before(scores[u], u, st, t)) ++ahead;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
-      evict = ahead >= n_keep;
+        for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
+        evict = ahead >= n_keep;
+      }
+      if (lane == 0) v.prune_rank[t] = evict;
     }
-    if (lane == 0) v.prune_rank[t] = evict;
+    __syncthreads();
+    // ---- 3. evicted ids, ascending
+    int n_list = 0;
+    for (int base = 0; base < T; base += blockDim.x) {
+      const int t = base + threadIdx.x;
+      const int f = t < T ? v.prune_rank[t] : 0;
+      int chunk_total;
+      const int at = block_excl_scan(f, s_warp, &chunk_total);
+      if (f) { v.prune_list[n_list + at] = t; pruned_ids_out[n_list + at] = t; }
+      n_list += chunk_total;
+    }
+    if (threadIdx.x == 0) { *n_pruned_out = n_list; v.counters[C_PRUNE_N] = n_list; }
+    __threadfence();
   }
-  __syncthreads();
-  // ---- 3. evicted ids, ascending
-  int n_list = 0;
-  for (int base = 0; base < T; base += blockDim.x) {
-    const int t = base + threadIdx.x;
-    const int f = t < T ? v.prune_rank[t] : 0;
-    int chunk_total;
-    const int at = block_excl_scan(f, s_warp, &chunk_total);
-    if (f) { v.prune_list[n_list + at] = t; pruned_ids_out[n_list + at] = t; }
-    n_list += chunk_total;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) *n_pruned_out = n_list;
+  cluster.sync();
   // ---- 4. release
-  release_listed(v, g, n_list, unscored, s_warp);
+  release_listed_cluster(v, g, __ldcg(&v.counters[C_PRUNE_N]), unscored, s_warp);
 }
 
-__global__ void __launch_bounds__(kPruneThreads)
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kPruneThreads, 1)
 release_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, float unscored) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   __shared__ int s_warp[33];
-  __shared__ int s_n;
   // keep the valid, live ids in the order given
-  if (threadIdx.x == 0) {
+  if (cluster.block_rank() == 0 && threadIdx.x == 0) {
     int k = 0;
     for (int i = 0; i < n; ++i) {
       const int t = ids[i];
       if (t < 0 || t >= g.max_traces || !v.live[t]) { flag_error(v.counters, STEP_ERR_BAD_TRACE); continue; }
       v.prune_list[k++] = t;
     }
-    s_n = k;
+    v.counters[C_PRUNE_N] = k;
+    __threadfence();
   }
-  __syncthreads();
-  release_listed(v, g, s_n, unscored, s_warp);
+  cluster.sync();
+  release_listed_cluster(v, g, __ldcg(&v.counters[C_PRUNE_N]), unscored, s_warp);
 }
 
 }  // namespace
@@ -204,7 +119,7 @@ int prune_if_saturated(step_pool* pool, const float* scores, float threshold, fl
   if (!pool || !pruned_ids_out || !n_pruned_out) return STEP_ERR_INVALID_ARG;
   if (!(threshold > 0.f) || threshold > 1.f) return STEP_ERR_INVALID_ARG;
   if (isnan(keep_frac) || keep_frac == 0.f || keep_frac > 1.f) return STEP_ERR_INVALID_ARG;
-  prune_kernel<<<1, kPruneThreads, 0, (cudaStream_t)stream>>>(pool->v, geo_of(pool), scores, threshold, keep_frac,
+  prune_kernel<<<kClusterCtas, kPruneThreads, 0, (cudaStream_t)stream>>>(pool->v, geo_of(pool), scores, threshold, keep_frac,
                                                               pool->cfg.unscored_score, pruned_ids_out, n_pruned_out);
   return launch_ok();
 }
@@ -213,7 +128,7 @@ int kv_pool_release_traces(step_pool* pool, const int32_t* trace_ids, int n, voi
   if (!pool || n < 0) return STEP_ERR_INVALID_ARG;
   if (n == 0) return STEP_OK;
   if (!trace_ids || n > pool->cfg.max_traces) return STEP_ERR_INVALID_ARG;
-  release_kernel<<<1, kPruneThreads, 0, (cudaStream_t)stream>>>(pool->v, geo_of(pool), trace_ids, n,
+  release_kernel<<<kClusterCtas, kPruneThreads, 0, (cudaStream_t)stream>>>(pool->v, geo_of(pool), trace_ids, n,
                                                                 pool->cfg.unscored_score);
   return launch_ok();
 }
