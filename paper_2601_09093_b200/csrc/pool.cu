@@ -52,6 +52,12 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.score_part = take((rows + kScoreFoldRows - 1) / kScoreFoldRows * T * 8);
   l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
   l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
+  l.final_score = take(T * 4);
+  l.answer = take(T * 4);
+  l.finished = take(T);
+  l.it_ids = take(T * 4);
+  l.it_fin = take(T * 4);
+  l.it_pruned = take(T * 4);
   l.total = off;
   return l;
 }
@@ -69,6 +75,7 @@ __global__ void init_meta_kernel(DevViews v, Geo g, float unscored) {
   for (size_t i = tid; i < (size_t)g.max_traces; i += stride) {
     v.seq_lens[i] = 0; v.live[i] = 0; v.score_sum[i] = 0.f; v.score_cnt[i] = 0;
     v.trace_scores[i] = unscored; v.append_base[i] = -1;
+    v.final_score[i] = 0.f; v.answer[i] = -1; v.finished[i] = 0;
   }
   for (size_t i = tid; i < (size_t)g.num_blocks; i += stride) {
     v.refcount[i] = 0; v.claim[i] = -1;
@@ -141,15 +148,19 @@ __global__ void fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, con
 
 // ---------------------------------------------------------------- append_kv
 // Phase 1 (one CTA): decide, in list order, which traces get their pages; pop blocks.
-__global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, int n_tokens) {
+// n_dev (may be null): only the first min(n, *n_dev) listed traces take part; the rest are passed over in silence.
+__global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, int n_tokens,
+                                    const int32_t* __restrict__ n_dev) {
   extern __shared__ int sm[];
+  const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
   int* s_need = sm;            // pages wanted, or -1 if the trace is skipped
   int* s_off = sm + n;         // pops that precede this trace's
   int* s_have = sm + 2 * n;
   __shared__ int s_fc;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    const int t = ids[i];
     int need = -1, have = 0;
+    if (i >= n_eff) { s_need[i] = need; s_have[i] = have; continue; }
+    const int t = ids[i];
     if (t < 0 || t >= g.max_traces || !v.live[t]) {
       flag_error(v.counters, STEP_ERR_BAD_TRACE);
     } else {
@@ -180,8 +191,8 @@ __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   for (int i = warp; i < n; i += nwarps) {
     const int need = s_need[i];
-    const int t = ids[i];
     if (need < 0) { if (lane == 0) v.append_base[i] = -1; continue; }
+    const int t = ids[i];
     int32_t* row = v.block_table + (size_t)t * g.max_pages;
     for (int p = lane; p < need; p += 32) {
       const int b = v.free_list[fc - 1 - s_off[i] - p];
@@ -199,7 +210,7 @@ __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict
 // Phase 2: one thread moves one 16-byte chunk of a new K or V row into its page.
 __global__ void append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ knew,
                                     const uint4* __restrict__ vnew, const int32_t* __restrict__ ids,
-                                    int n, int n_tokens, int cpr, int cpe) {
+                                    int n, int n_tokens, int cpr, int cpe, int src_by_id) {
   const size_t per_kv = (size_t)n * n_tokens * g.L * g.Hkv * cpr;
   const size_t total = per_kv * 2;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -217,7 +228,9 @@ __global__ void append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, c
     const int b = v.block_table[(size_t)t * g.max_pages + page];
     const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
     const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
-    kv[e / cpe + cdst] = (which ? vnew : knew)[src];
+    // the new rows are laid out [row, token, layer, head, chunk]; row = position in the list, or the trace id
+    const size_t from = src_by_id ? ((((size_t)t * n_tokens + j) * g.L + layer) * g.Hkv + head) * cpr + c : src;
+    kv[e / cpe + cdst] = (which ? vnew : knew)[from];
   }
 }
 
@@ -303,6 +316,9 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
   v.score_part = (float2*)(m + lay.score_part);
   v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o);
+  v.final_score = (float*)(m + lay.final_score); v.answer = (int32_t*)(m + lay.answer);
+  v.finished = (uint8_t*)(m + lay.finished); v.it_ids = (int32_t*)(m + lay.it_ids);
+  v.it_fin = (int32_t*)(m + lay.it_fin); v.it_pruned = (int32_t*)(m + lay.it_pruned);
   int st = kv_pool_reset(p, nullptr);
   if (st == STEP_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = STEP_ERR_CUDA;
   if (st != STEP_OK) { delete p; return st; }
@@ -350,24 +366,34 @@ int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const voi
 
 int append_kv(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
               const void* v_new, void* stream) {
+  return stepk::append_kv_impl(pool, trace_ids, n, n_tokens, k_new, v_new, nullptr, 0, (cudaStream_t)stream);
+}
+
+}  // extern "C"
+
+int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
+                          const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s) {
   if (!pool || n < 0 || n_tokens < 0) return STEP_ERR_INVALID_ARG;
   if (n == 0 || n_tokens == 0) return STEP_OK;
   if (!trace_ids || !k_new || !v_new) return STEP_ERR_INVALID_ARG;
   if (n > pool->cfg.max_traces) return STEP_ERR_INVALID_ARG;   // ids must be distinct
   Geo g = geo_of(pool);
-  cudaStream_t s = (cudaStream_t)stream;
   const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
   const size_t row_chunks = (size_t)n_tokens * g.L * g.Hkv * cpr;   // 16-byte chunks of K (or V) per trace
   constexpr int kListChunk = 4096;                                  // traces per launch (shared-memory scan)
   for (int off = 0; off < n; off += kListChunk) {
     const int m = n - off < kListChunk ? n - off : kListChunk;
-    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens);
+    if (n_dev && off > 0) return STEP_ERR_INVALID_ARG;              // a device-side count covers one launch only
+    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens, n_dev);
+    const size_t src_off = src_by_id ? 0 : row_chunks * off;
     append_write_kernel<<<grid_for(row_chunks * m * 2, 256, pool->num_sms), 256, 0, s>>>(
-        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + row_chunks * off,
-        (const uint4*)v_new + row_chunks * off, trace_ids + off, m, n_tokens, cpr, cpe);
+        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off,
+        (const uint4*)v_new + src_off, trace_ids + off, m, n_tokens, cpr, cpe, src_by_id);
   }
   return launch_ok();
 }
+
+extern "C" {
 
 int kv_pool_stats(step_pool* pool, int* used, int* free_, int* total, int* live_traces, void* stream) {
   if (!pool) return STEP_ERR_INVALID_ARG;

@@ -41,15 +41,11 @@ template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return
 // mask_out if it is given.  An id outside the vocabulary ends no step and is flagged.
 constexpr int kRowsPerThread = 8;
 
-struct FlagSource {
-  const uint8_t* mask;       // [M], or nullptr
-  const int32_t* tokens;     // [M], or nullptr
-  const uint8_t* table;      // [vocab]
-  int vocab;
-  uint8_t* mask_out;         // [M], or nullptr
-};
-
 __device__ inline bool row_flag(const FlagSource& f, int i, int32_t* counters) {
+  if (f.live && !f.live[i]) {
+    if (f.mask_out) f.mask_out[i] = 0;
+    return false;
+  }
   if (!f.tokens) return f.mask[i] != 0;
   const int id = f.tokens[i];
   bool e = false;
@@ -242,9 +238,6 @@ step_end_kernel(FlagSource src, int M, int32_t* counters) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < M; i += gridDim.x * blockDim.x) row_flag(src, i, counters);
 }
 
-int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
-                     const scorer_weights* w, float* step_scores_out, void* stream);
-
 }  // namespace
 
 extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* boundary_mask,
@@ -253,7 +246,7 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
   if (!pool || M < 0 || !w) return STEP_ERR_INVALID_ARG;
   if (M == 0) return STEP_OK;
   if (!boundary_mask) return STEP_ERR_INVALID_ARG;
-  FlagSource src{boundary_mask, nullptr, nullptr, 0, nullptr};
+  FlagSource src{boundary_mask, nullptr, nullptr, 0, nullptr, nullptr};
   return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
 }
 
@@ -264,7 +257,7 @@ extern "C" int score_steps_tokens(step_pool* pool, const void* hidden, const int
   if (!pool || M < 0 || !w) return STEP_ERR_INVALID_ARG;
   if (M == 0) return STEP_OK;
   if (!token_ids || !step_end_table || vocab < 1) return STEP_ERR_INVALID_ARG;
-  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out};
+  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out, nullptr};
   return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
 }
 
@@ -273,7 +266,7 @@ extern "C" int detect_step_ends(step_pool* pool, const int32_t* token_ids, int M
   if (!pool || M < 0) return STEP_ERR_INVALID_ARG;
   if (M == 0) return STEP_OK;
   if (!token_ids || !step_end_table || vocab < 1 || !boundary_mask_out) return STEP_ERR_INVALID_ARG;
-  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out};
+  FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out, nullptr};
   int ctas = (M + 255) / 256;
   if (ctas > pool->num_sms * 8) ctas = pool->num_sms * 8;
   step_end_kernel<<<ctas, 256, 0, (cudaStream_t)stream>>>(src, M, pool->v.counters);
@@ -300,10 +293,8 @@ extern "C" int step_end_table_from_vocab(const char* const* token_text, const in
   return STEP_OK;
 }
 
-namespace {
-
-int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
-                     const scorer_weights* w, float* step_scores_out, void* stream) {
+int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
+                            const scorer_weights* w, float* step_scores_out, void* stream) {
   if (!hidden || !step_scores_out) return STEP_ERR_INVALID_ARG;
   if (!w->W1 || !w->b1 || !w->w2 || w->D < 1 || w->m < 1) return STEP_ERR_INVALID_ARG;
   if (w->dtype != STEP_BF16 && w->dtype != STEP_FP32) return STEP_ERR_INVALID_ARG;
@@ -322,6 +313,7 @@ int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const 
     if (part.mask) part.mask += off;
     if (part.tokens) part.tokens += off;
     if (part.mask_out) part.mask_out += off;
+    if (part.live) part.live += off;
     score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, part, Mc, step_scores_out + off,
                                                        tc_min_rows, w->m, pool->num_sms);
     // the CUDA-core kernel only ever sees launches with fewer than tc_min_rows boundary rows
@@ -350,8 +342,6 @@ int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const 
   }
   return launch_ok();
 }
-
-}  // namespace
 
 extern "C" int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows) {
   if (!pool || mode < -1 || mode > 1 || tc_min_rows < 0) return STEP_ERR_INVALID_ARG;

@@ -28,7 +28,9 @@ constexpr int kScoreFoldRows = 512;    // listed rows one CTA of the scorer's fi
 // number of hidden units (UMMA N) each CTA of the tensor-core kernel covers.  C_SCORE_SLICES:
 // how many partial sums per row the MLP kernels leave in score_z.
 enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4,
-               C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_SCORE_TICKET = 7, C_NUM = 64 };
+               C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_SCORE_TICKET = 7,
+               // Algorithm 1 driver: live / finishing traces of the current iteration, running totals
+               C_IT_NLIVE = 8, C_IT_NFIN = 9, C_N_FINISHED = 10, C_N_EVICTED = 11, C_IT_NPRUNED = 12, C_NUM = 64 };
 
 struct MetaLayout {
   size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;
@@ -36,6 +38,7 @@ struct MetaLayout {
   size_t append_base, prune_rank, prune_list, prune_off;
   size_t score_idx, score_z, score_part;
   size_t attn_ml, attn_o;
+  size_t final_score, answer, finished, it_ids, it_fin, it_pruned;
   size_t total;
 };
 
@@ -46,6 +49,8 @@ struct DevViews {
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
   int32_t* score_idx; float* score_z; float2* score_part;
   float* attn_ml; float* attn_o;
+  float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
+  int32_t* it_ids; int32_t* it_fin; int32_t* it_pruned;       // per-iteration lists of the Algorithm 1 driver
 };
 
 }  // namespace stepk
@@ -105,6 +110,26 @@ __device__ inline void flag_error(int32_t* counters, int code) {
   } while (0)
 
 inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? STEP_OK : STEP_ERR_CUDA; }
+
+// ---- pieces the Algorithm 1 driver (algorithm1.cu) chains together
+// append_kv with two extras: *n_dev (device, may be null) caps the number of listed traces on the device, and
+// src_by_id makes trace t read row t of k_new / v_new instead of row (position in the list).
+int append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
+                   const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s);
+
+// Where score_steps takes a row's step-end flag from: mask[i], or table[tokens[i]] (a token ends a step if its
+// text contains two newlines in a row; the table records that per vocabulary entry).  live (may be null)
+// additionally requires live[i] != 0 - for callers whose row i is trace i.
+struct FlagSource {
+  const uint8_t* mask;       // [M], or nullptr
+  const int32_t* tokens;     // [M], or nullptr
+  const uint8_t* table;      // [vocab]
+  int vocab;
+  uint8_t* mask_out;         // [M], or nullptr
+  const uint8_t* live;       // [M], or nullptr
+};
+int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
+                     const scorer_weights* w, float* step_scores_out, void* stream);
 
 // ---- tensor-core scorer (scorer_tc.cu)
 // True if the tcgen05 kernel covers this scorer shape and these pointers.
