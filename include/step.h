@@ -195,7 +195,90 @@ int prune_if_saturated(step_pool* pool, const float* scores, float threshold, fl
 /* A trace that finished on its own gives its KV back (same reclaim as an eviction). */
 int kv_pool_release_traces(step_pool* pool, const int32_t* trace_ids, int n, void* stream);
 
+/* ---- Algorithm 1 as a loop over device-resident state ----
+ * The model's forward pass is outside this library, so NextToken(t) -> (x, h) is represented by what goes in
+ * and comes out of it: per iteration the caller supplies, for every trace, the sampled token x, the new K/V
+ * rows, the queries of the layers whose attention is to be run and the last-layer hidden state h.  In all of
+ * these ROW i IS TRACE i (the traces are ids 0 .. n_traces-1 of the pool, forked before the first iteration),
+ * and rows of traces that are no longer live are passed over on the device, so the host never needs to know
+ * who is live.  One memory-trigger check is made per iteration, after the iteration's cache writes. */
+
+/* A trace that completed: its current score_t and its answer id (>= 0) are kept for the vote, then its KV is
+ * released as for an eviction.  trace_ids, answers: [n] device; a trace whose answer is negative, or all of
+ * them if answers is NULL, completes without taking part in the vote.  Ids must be distinct; invalid or dead
+ * ids are flagged (STEP_ERR_BAD_TRACE) and skipped. */
+int kv_pool_finish_traces(step_pool* pool, const int32_t* trace_ids, const int32_t* answers, int n, void* stream);
+
+/* WeightedVote(T, {score_t}) (Algorithm 1, last line; Sec. 3.3): over the completed traces, the answer with the
+ * largest sum of final trace scores; equal sums go to the smaller answer id.  Evicted traces do not vote.
+ * answer_out [1] int32 (-1 if no trace completed), weight_out [1] float (may be NULL), n_finished_out [1] int32
+ * (may be NULL): device pointers. */
+int weighted_vote(step_pool* pool, int32_t* answer_out, float* weight_out, int32_t* n_finished_out, void* stream);
+
+typedef struct {
+  int n_traces;                       /* rows of every per-trace input below                                      */
+  const int32_t* token_ids;           /* [n] the token each trace sampled                                         */
+  int eos_token;                      /* a live trace that sampled it completes in this iteration                 */
+  const uint8_t* step_end_table;      /* [vocab] see step_end_table_from_vocab                                    */
+  int vocab;
+  const int32_t* answers;             /* [n] answer id trace i reports if it completes now (may be NULL)          */
+  int n_layers_attention;             /* decode_attention is run for layers 0 .. this-1 (0: none)                 */
+  const void* q;                      /* [n_layers_attention, n, num_q_heads, head_dim] pool dtype                */
+  const void* k_new; const void* v_new; /* [n, 1, num_layers, num_kv_heads, head_dim] pool dtype                  */
+  const void* hidden;                 /* [n, D] scorer dtype                                                      */
+  void* attn_out;                     /* [n_layers_attention, n, num_q_heads, head_dim] fp32                      */
+  float* step_scores_out;             /* [n] as score_steps                                                       */
+  uint8_t* boundary_mask_out;         /* [n] step-end flags of the live rows (may be NULL)                        */
+  float* trace_scores_out;            /* [n] score_t of every trace right after this iteration's scoring, i.e. what
+                                         completion records and eviction ranks by (may be NULL)                    */
+  const scorer_weights* scorer;
+  float threshold, keep_frac;         /* as prune_if_saturated; keep_frac < 0 with threshold 1 is the paper's rule */
+  int max_evictions;                  /* the trigger is tested, and the rule applied, up to this many times in a row
+                                         (0 or 1: once); each further test sees the pool the last eviction left      */
+  int32_t* pruned_ids_out;            /* [max_traces], may be NULL; holds the last test's evictions               */
+  int32_t* n_pruned_out;              /* [1], may be NULL                                                         */
+} step_iteration;
+
+/* One iteration of the while loop of Algorithm 1 for all traces, chained on the stream with no host round trip:
+ * append_kv of the live traces' new token -> decode_attention per layer -> step-end detection + score_steps ->
+ * completion (kv_pool_finish_traces) of the live traces whose token is eos_token -> prune_if_saturated on the
+ * pool's running means (max_evictions times: with the paper's one-eviction rule a single eviction may not free
+ * enough blocks for the next step when many traces reach a page boundary together).  All pointers are device pointers except `it` and it->scorer (host structs). */
+int algorithm1_iteration(step_pool* pool, const step_iteration* it, void* stream);
+
+typedef struct {
+  int n_traces, max_iterations;
+  const int32_t* token_ids;           /* [max_iterations, n] sampled tokens, iteration-major                      */
+  int eos_token;
+  const uint8_t* step_end_table; int vocab;
+  const int32_t* answers;             /* [n]                                                                      */
+  int ring;                           /* the per-iteration tensors below hold `ring` slots; iteration i uses i % ring */
+  int n_layers_attention;
+  const void* q;                      /* [ring, n_layers_attention, n, num_q_heads, head_dim]                     */
+  const void* k_new; const void* v_new; /* [ring, n, 1, num_layers, num_kv_heads, head_dim]                       */
+  const void* hidden;                 /* [ring, n, D]                                                             */
+  void* attn_out;                     /* [n_layers_attention, n, num_q_heads, head_dim] fp32, overwritten each iteration */
+  float* step_scores_out;             /* [n]                                                                      */
+  const scorer_weights* scorer;
+  float threshold, keep_frac;
+  int max_evictions;                  /* as in step_iteration                                                     */
+  int check_every;                    /* the host asks for the number of live traces every this many iterations   */
+  float* score_history;               /* [max_iterations, n] score_t after each iteration's scoring, or NULL      */
+} step_run_args;
+
+typedef struct {
+  int iterations;                     /* iterations executed                                                      */
+  int answer; float answer_weight;    /* the vote's result (-1 if no trace completed)                             */
+  int n_finished, n_evicted, live_left;
+} step_run_result;
+
+/* The whole loop: iterations until no trace is live (checked every check_every iterations; iterations with no
+ * live trace do nothing) or max_iterations, then the weighted vote.  res is a HOST struct; synchronises. */
+int algorithm1_run(step_pool* pool, const step_run_args* args, step_run_result* res, void* stream);
+
 /* ---- accessors for tests and benchmarks ---- */
+/* Vote state: final_score [max_traces] f32, answer [max_traces] i32, finished [max_traces] u8 (device). */
+int kv_pool_vote_views(step_pool* pool, float** final_score, int32_t** answer, uint8_t** finished);
 /* Host ints; synchronises the stream. */
 int kv_pool_stats(step_pool* pool, int* used, int* free_, int* total, int* live_traces, void* stream);
 /* Device pointers into meta_storage (any may be NULL):

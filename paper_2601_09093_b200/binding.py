@@ -41,6 +41,30 @@ class scorer_weights(C.Structure):
                 ("D", C.c_int), ("m", C.c_int), ("dtype", C.c_int)]
 
 
+class step_iteration(C.Structure):
+    _fields_ = [("n_traces", C.c_int), ("token_ids", C.c_void_p), ("eos_token", C.c_int),
+                ("step_end_table", C.c_void_p), ("vocab", C.c_int), ("answers", C.c_void_p),
+                ("n_layers_attention", C.c_int), ("q", C.c_void_p), ("k_new", C.c_void_p), ("v_new", C.c_void_p),
+                ("hidden", C.c_void_p), ("attn_out", C.c_void_p), ("step_scores_out", C.c_void_p),
+                ("boundary_mask_out", C.c_void_p), ("trace_scores_out", C.c_void_p), ("scorer", C.POINTER(scorer_weights)),
+                ("threshold", C.c_float), ("keep_frac", C.c_float), ("max_evictions", C.c_int),
+                ("pruned_ids_out", C.c_void_p), ("n_pruned_out", C.c_void_p)]
+
+
+class step_run_args(C.Structure):
+    _fields_ = [("n_traces", C.c_int), ("max_iterations", C.c_int), ("token_ids", C.c_void_p), ("eos_token", C.c_int),
+                ("step_end_table", C.c_void_p), ("vocab", C.c_int), ("answers", C.c_void_p), ("ring", C.c_int),
+                ("n_layers_attention", C.c_int), ("q", C.c_void_p), ("k_new", C.c_void_p), ("v_new", C.c_void_p),
+                ("hidden", C.c_void_p), ("attn_out", C.c_void_p), ("step_scores_out", C.c_void_p),
+                ("scorer", C.POINTER(scorer_weights)), ("threshold", C.c_float), ("keep_frac", C.c_float),
+                ("max_evictions", C.c_int), ("check_every", C.c_int), ("score_history", C.c_void_p)]
+
+
+class step_run_result(C.Structure):
+    _fields_ = [("iterations", C.c_int), ("answer", C.c_int), ("answer_weight", C.c_float),
+                ("n_finished", C.c_int), ("n_evicted", C.c_int), ("live_left", C.c_int)]
+
+
 _lib = None
 
 
@@ -75,6 +99,11 @@ def lib():
     L.kv_pool_last_error.argtypes = [vp, C.POINTER(C.c_uint), vp]
     L.kv_pool_read_kv.argtypes = [vp, i, i, vp, i, vp, vp, vp]
     L.kv_pool_set_attention_config.argtypes = [vp, i, i]
+    L.kv_pool_finish_traces.argtypes = [vp, vp, vp, i, vp]
+    L.weighted_vote.argtypes = [vp, vp, vp, vp, vp]
+    L.kv_pool_vote_views.argtypes = [vp] + [C.POINTER(vp)] * 3
+    L.algorithm1_iteration.argtypes = [vp, C.POINTER(step_iteration), vp]
+    L.algorithm1_run.argtypes = [vp, C.POINTER(step_run_args), C.POINTER(step_run_result), vp]
     L.kv_pool_set_scorer_config.argtypes = [vp, i, i]
     L.kv_pool_score_launch_info.argtypes = [vp, ip, ip, vp]
     _lib = L
@@ -245,6 +274,68 @@ class KVPool:
         _check("kv_pool_read_kv", lib().kv_pool_read_kv(self.handle, layer, kv_head, _ptr(block_row), seq_len, _ptr(k),
                                                         _ptr(v), _stream(stream)))
         return k, v
+
+    # ---- Algorithm 1 as a loop
+    def finish_traces(self, trace_ids, answers, stream=None):
+        _check("kv_pool_finish_traces", lib().kv_pool_finish_traces(self.handle, _ptr(trace_ids), _ptr(answers),
+                                                                    trace_ids.numel(), _stream(stream)))
+
+    def weighted_vote(self, stream=None):
+        """Returns device tensors (answer [1] int32, weight [1] float32, n_finished [1] int32); no sync."""
+        a = torch.empty(1, dtype=torch.int32, device=self.device)
+        w = torch.empty(1, dtype=torch.float32, device=self.device)
+        n = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check("weighted_vote", lib().weighted_vote(self.handle, _ptr(a), _ptr(w), _ptr(n), _stream(stream)))
+        return a, w, n
+
+    def vote_views(self):
+        p = [C.c_void_p() for _ in range(3)]
+        _check("kv_pool_vote_views", lib().kv_pool_vote_views(self.handle, *[C.byref(x) for x in p]))
+        T = self.max_traces
+        return dict(final_score=self._view(p[0].value, T, torch.float32), answer=self._view(p[1].value, T, torch.int32),
+                    finished=self._view(p[2].value, T, torch.uint8))
+
+    def algorithm1_iteration(self, token_ids, eos_token, step_end_table, answers, q, k_new, v_new, hidden, weights,
+                             threshold, keep_frac, max_evictions=1, attn_out=None, step_scores_out=None,
+                             boundary_mask_out=None, trace_scores_out=None, pruned_ids_out=None, n_pruned_out=None,
+                             stream=None):
+        """One iteration of the loop for traces 0 .. n-1 (row i of every input is trace i); no sync.
+        q: [layers, n, Hq, d] or None (no attention)."""
+        n = token_ids.numel()
+        La = 0 if q is None else q.shape[0]
+        if La and attn_out is None:
+            attn_out = torch.empty((La, n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=self.device)
+        if step_scores_out is None:
+            step_scores_out = torch.empty(n, dtype=torch.float32, device=self.device)
+        it = step_iteration(n_traces=n, token_ids=token_ids.data_ptr(), eos_token=eos_token,
+                            step_end_table=step_end_table.data_ptr(), vocab=step_end_table.numel(),
+                            answers=_ptr(answers).value, n_layers_attention=La, q=_ptr(q).value, k_new=k_new.data_ptr(),
+                            v_new=v_new.data_ptr(), hidden=hidden.data_ptr(), attn_out=_ptr(attn_out).value,
+                            step_scores_out=step_scores_out.data_ptr(), boundary_mask_out=_ptr(boundary_mask_out).value,
+                            trace_scores_out=_ptr(trace_scores_out).value, scorer=C.pointer(weights.struct), threshold=threshold, keep_frac=keep_frac,
+                            max_evictions=max_evictions, pruned_ids_out=_ptr(pruned_ids_out).value, n_pruned_out=_ptr(n_pruned_out).value)
+        _check("algorithm1_iteration", lib().algorithm1_iteration(self.handle, C.byref(it), _stream(stream)))
+        return attn_out, step_scores_out
+
+    def algorithm1_run(self, token_ids, eos_token, step_end_table, answers, q, k_new, v_new, hidden, weights, threshold,
+                       keep_frac, max_evictions=1, check_every=16, attn_out=None, score_history=None, stream=None):
+        """The whole loop.  token_ids: [max_iterations, n]; q: [ring, layers, n, Hq, d] or None;
+        k_new, v_new: [ring, n, 1, L, Hkv, d]; hidden: [ring, n, D].  Returns the result as a dict (synchronises)."""
+        max_it, n = token_ids.shape
+        ring = k_new.shape[0]
+        La = 0 if q is None else q.shape[1]
+        if La and attn_out is None:
+            attn_out = torch.empty((La, n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=self.device)
+        scores = torch.empty(n, dtype=torch.float32, device=self.device)
+        a = step_run_args(n_traces=n, max_iterations=max_it, token_ids=token_ids.data_ptr(), eos_token=eos_token,
+                          step_end_table=step_end_table.data_ptr(), vocab=step_end_table.numel(), answers=_ptr(answers).value,
+                          ring=ring, n_layers_attention=La, q=_ptr(q).value, k_new=k_new.data_ptr(), v_new=v_new.data_ptr(),
+                          hidden=hidden.data_ptr(), attn_out=_ptr(attn_out).value, step_scores_out=scores.data_ptr(),
+                          scorer=C.pointer(weights.struct), threshold=threshold, keep_frac=keep_frac, max_evictions=max_evictions, check_every=check_every,
+                          score_history=_ptr(score_history).value)
+        r = step_run_result()
+        _check("algorithm1_run", lib().algorithm1_run(self.handle, C.byref(a), C.byref(r), _stream(stream)))
+        return {k: getattr(r, k) for k, _ in step_run_result._fields_}
 
     def set_attention_config(self, grid_ctas=0, fast_path=0):
         _check("kv_pool_set_attention_config", lib().kv_pool_set_attention_config(self.handle, grid_ctas, fast_path))

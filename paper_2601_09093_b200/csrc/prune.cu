@@ -82,7 +82,7 @@ prune_kernel(DevViews v, Geo g, const float* __restrict__ scores_in, float thres
       if (f) { v.prune_list[n_list + at] = t; pruned_ids_out[n_list + at] = t; }
       n_list += chunk_total;
     }
-    if (threadIdx.x == 0) { *n_pruned_out = n_list; v.counters[C_PRUNE_N] = n_list; }
+    if (threadIdx.x == 0) { *n_pruned_out = n_list; v.counters[C_PRUNE_N] = n_list; v.counters[C_N_EVICTED] += n_list; }
     __threadfence();
   }
   cluster.sync();
