@@ -305,11 +305,11 @@ def run_ours(args):
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
                      "traffic": None if ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE is None else algo_bytes * ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE,
                      "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the one-layer 64-trace workload, scaled by algorithmic bytes",
-                     "kernel": "decode_attention (attn_mma_kernel + attn_merge_kernel), one layer",
+                     "kernel": "decode_attention (attn_mma_kernel, split partials merged in the same launch), one layer",
                      "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": attn_avg_ms,
                      "min_launch_ms": float(np.min(attn_ms)), "launches_timed": len(attn_ms)},
         "kv_gbs": achieved, "attention_share_of_step": float(np.sum(attn_ms)) / ms_total,
-        "gpu_launches": K * (2 + 2 * L + 3 + 1), "clocks": clocks,
+        "gpu_launches": K * (2 + L + 3 + 1), "clocks": clocks,
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
     if e2e:

@@ -131,17 +131,18 @@ int decode_attention(step_pool* pool, int layer, const void* q,
  * cudaFree and calls no allocating routine.
  *
  * Limits (fixed by that array): bf16 pools with head_dim 128 and page_size 16 only (else
- * STEP_ERR_INVALID_ARG); num_q_heads / num_kv_heads <= 8 and n <= 2048, else STEP_ERR_CAPACITY with
- * nothing launched.  The launch uses at most 148 CTAs whatever kv_pool_set_attention_config says.
+ * STEP_ERR_INVALID_ARG); num_q_heads / num_kv_heads <= 8, n <= 2048 and n * num_kv_heads <= 16384, else
+ * STEP_ERR_CAPACITY with nothing launched.  The launch uses at most 148 CTAs whatever kv_pool_set_attention_config says.
  * The pool's device must be the current device.
  *
  * First use on a device: the first call on each device looks up the array's device address
  * (cudaGetSymbolAddress) before it launches.  Make that first call outside any stream capture.
  *
  * Sharing: all calls on a device - from every pool and every stream - use the same array, and it
- * keeps whatever the previous call left.  Nothing in it has to start at zero (each call writes every
- * partial before it reads it), but two calls that overlap in time on the GPU race on it: keep
- * calls of this entry point ordered, e.g. on one stream. */
+ * keeps whatever the previous call left.  The partials need no clearing (each call writes every partial
+ * before it reads it); the small ticket counters in it must be zero when a call starts, which they are: they
+ * start as zero bits and every call that runs to its end puts them back to zero.  Two calls that overlap in
+ * time on the GPU race on the array: keep calls of this entry point ordered, e.g. on one stream. */
 int decode_attention_static(step_pool* pool, int layer, const void* q,
                             const int32_t* block_table, const int32_t* seq_lens, int n,
                             void* out, void* stream);

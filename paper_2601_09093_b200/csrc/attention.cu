@@ -19,8 +19,9 @@
 //        heads on the M axis, ldmatrix (plain for K, transposed for V) feeding the B operand;
 //      - running (max, sum) softmax state per head in fp32, exp2 with the scale folded in;
 //      - a partition that holds a whole (trace, head) sequence writes the output directly;
-//        otherwise it writes an (m, l, o) partial (at most two per warp) and attn_merge_kernel
-//        combines the partials of each split (trace, head).
+//        otherwise it writes an (m, l, o) partial (at most two per warp) and takes a ticket on that
+//        sequence's counter; the warp that draws the last ticket combines the sequence's partials
+//        and writes the output (no second kernel, no waiting: whoever is last does the work).
 #include "step_internal.cuh"
 
 #include <math.h>
@@ -119,6 +120,7 @@ struct AttnArgs {
   float* out;
   float* ws_ml;                    // [partition][2][G][2]
   float* ws_o;                     // [partition][2][G][kD]
+  int32_t* seg_cnt;                // [n][Hkv] tickets of the split sequences; zero between launches
   int32_t* counters;
   int n, Hq, Hkv, G, max_pages, num_blocks;
   float scale_log2;
@@ -244,6 +246,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+
+  // traces without any position get zeros (CTAs take the traces round-robin)
+  for (int t = blockIdx.x; t < n; t += gridDim.x)
+    if (s_cum[t + 1] == s_cum[t])
+      for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) a.out[(size_t)t * a.Hq * kD + k] = 0.f;
 
   const long long total = (long long)Hkv * s_cum[n];
   const int n_part = gridDim.x * kWarps;
@@ -456,6 +463,37 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
           for (int dt = 0; dt < 16; ++dt)
             *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2], o_acc[dt][3]);
         }
+        // publish the partial, take a ticket; the last of the sequence's partitions to arrive merges them all
+        __threadfence();
+        __syncwarp();
+        const long long seg_start = (long long)Hkv * s_cum[cc.t] + (long long)cc.h * cc.np;
+        const int w_first = (int)(seg_start / W), w_last = (int)((seg_start + cc.np - 1) / W);
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&a.seg_cnt[cc.t * Hkv + cc.h], 1);
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+        if (ticket == w_last - w_first) {
+          if (lane == 0) a.seg_cnt[cc.t * Hkv + cc.h] = 0;             // ready for the next launch
+          __threadfence();
+          float* og = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
+          for (int g = 0; g < G; ++g) {
+            float M = -INFINITY;
+            for (int w = w_first; w <= w_last; ++w) {
+              const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
+              M = fmaxf(M, __ldcg(&a.ws_ml[(sl * G + g) * 2]));
+            }
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+            float den = 0.f;
+            for (int w = w_first; w <= w_last; ++w) {
+              const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
+              const float wgt = exp2f(__ldcg(&a.ws_ml[(sl * G + g) * 2]) - M);
+              den += wgt * __ldcg(&a.ws_ml[(sl * G + g) * 2 + 1]);
+              const float4 o4 = __ldcg(reinterpret_cast<const float4*>(a.ws_o + (sl * G + g) * kD) + lane);
+              num.x += wgt * o4.x; num.y += wgt * o4.y; num.z += wgt * o4.z; num.w += wgt * o4.w;
+            }
+            const float inv = 1.f / den;
+            reinterpret_cast<float4*>(og + (size_t)g * kD)[lane] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+          }
+        }
       }
       seg_open = false;
       seg_is_first = false;
@@ -471,60 +509,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
       mbar_wait_bounded(my_bar_u32 + s * 8, 0);
       mbar_wait_bounded(my_bar_u32 + s * 8, 1);
     }
-  }
-}
-
-// Combines the partials of every (trace, kv head) sequence that more than one partition touched,
-// and writes zeros for empty sequences.  grid (Hkv, n), kD threads.
-__global__ void __launch_bounds__(kD) attn_merge_kernel(AttnArgs a, int n_part) {
-  __shared__ int s_red[2][kD / 32];
-  const int h = blockIdx.x, t = blockIdx.y, n = a.n, G = a.G;
-  int before = 0, all = 0, mine = 0;
-  for (int u = threadIdx.x; u < n; u += blockDim.x) {
-    int S = a.seq_lens[u];
-    if (S < 0) S = 0;
-    int pages = (S + kP - 1) / kP;
-    if (pages > a.max_pages) pages = a.max_pages;
-    all += pages;
-    if (u < t) before += pages;
-    if (u == t) mine = pages;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    before += __shfl_xor_sync(0xffffffffu, before, o);
-    all += __shfl_xor_sync(0xffffffffu, all, o);
-    mine += __shfl_xor_sync(0xffffffffu, mine, o);
-  }
-  __shared__ int s_mine[kD / 32];
-  if ((threadIdx.x & 31) == 0) { s_red[0][threadIdx.x >> 5] = before; s_red[1][threadIdx.x >> 5] = all; s_mine[threadIdx.x >> 5] = mine; }
-  __syncthreads();
-  before = all = mine = 0;
-  for (int w = 0; w < kD / 32; ++w) { before += s_red[0][w]; all += s_red[1][w]; mine += s_mine[w]; }
-  const int np = mine;
-  float* ob = a.out + ((size_t)t * a.Hq + (size_t)h * G) * kD;
-  if (np == 0) {
-    for (int g = 0; g < G; ++g) ob[(size_t)g * kD + threadIdx.x] = 0.f;
-    return;
-  }
-  const long long total = (long long)a.Hkv * all;
-  const long long W = (total + n_part - 1) / n_part;
-  const long long start = (long long)a.Hkv * before + (long long)h * np;
-  const int w_first = (int)(start / W), w_last = (int)((start + np - 1) / W);
-  if (w_first == w_last) return;                       // written whole by one warp
-  for (int g = 0; g < G; ++g) {
-    float M = -INFINITY;
-    for (int w = w_first; w <= w_last; ++w) {
-      const size_t slot = (size_t)w * 2 + (start <= (long long)w * W ? 0 : 1);
-      M = fmaxf(M, a.ws_ml[(slot * G + g) * 2]);
-    }
-    float num = 0.f, den = 0.f;
-    for (int w = w_first; w <= w_last; ++w) {
-      const size_t slot = (size_t)w * 2 + (start <= (long long)w * W ? 0 : 1);
-      const float wgt = exp2f(a.ws_ml[(slot * G + g) * 2] - M);
-      den += wgt * a.ws_ml[(slot * G + g) * 2 + 1];
-      num += wgt * a.ws_o[(slot * G + g) * kD + threadIdx.x];
-    }
-    ob[(size_t)g * kD + threadIdx.x] = num / den;
   }
 }
 
@@ -545,7 +529,6 @@ int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
     kern<<<grid, kWarps * 32, smem, s>>>(a);
   }
-  attn_merge_kernel<<<dim3(a.Hkv, a.n), kD, 0, s>>>(a, grid * kWarps);
   return launch_ok();
 }
 
@@ -566,7 +549,7 @@ extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const
     a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
     a.q = (const __nv_bfloat16*)q;
     a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
-    a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.counters = pool->v.counters;
+    a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.seg_cnt = pool->v.attn_cnt; a.counters = pool->v.counters;
     a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
     return launch_mma<kWarpsDefault, kStagesDefault>(pool, a, s);
@@ -605,7 +588,8 @@ constexpr int kStaticMaxPartitions = 1184;   // 148 SMs x 8 warps
 constexpr int kStaticMaxG = 8;               // query heads per KV head
 constexpr size_t kStaticMlFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * 2;
 constexpr size_t kStaticOFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * kD;
-constexpr size_t kStaticScratchFloats = kStaticMlFloats + kStaticOFloats;
+constexpr int kStaticMaxSegs = 16384;        // (trace, KV head) sequences of one call: their ticket counters
+constexpr size_t kStaticScratchFloats = kStaticMlFloats + kStaticOFloats + kStaticMaxSegs;
 
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
@@ -637,7 +621,7 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   // only the shape the tensor-core kernel covers
   if (pool->cfg.dtype != STEP_BF16 || g.d != kD || g.P != kP || !pool->swizzle) return STEP_ERR_INVALID_ARG;
   // sizes beyond what the fixed scratch holds
-  if (g.G > kStaticMaxG || n > kMaxTracesFast) return STEP_ERR_CAPACITY;
+  if (g.G > kStaticMaxG || n > kMaxTracesFast || (long long)n * g.Hkv > kStaticMaxSegs) return STEP_ERR_CAPACITY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return STEP_ERR_CUDA;
   if (dev != pool->device) return STEP_ERR_INVALID_ARG;   // the pool's device must be current
@@ -652,6 +636,8 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   a.q = (const __nv_bfloat16*)q;
   a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
   a.ws_ml = scratch; a.ws_o = scratch + kStaticMlFloats; a.counters = pool->v.counters;
+  // the counters start as zero bits (static storage) and every launch leaves them zero again
+  a.seg_cnt = reinterpret_cast<int32_t*>(scratch + kStaticMlFloats + kStaticOFloats);
   a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
   const size_t smem = (size_t)kWarpsDefault * kStagesDefault * kPageBytes + (size_t)kWarpsDefault * kStagesDefault * 8 +
@@ -660,6 +646,5 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
   cudaStream_t s = (cudaStream_t)stream;
   kern<<<grid, kWarpsDefault * 32, smem, s>>>(a);
-  attn_merge_kernel<<<dim3(a.Hkv, a.n), kD, 0, s>>>(a, grid * kWarpsDefault);
   return launch_ok();
 }

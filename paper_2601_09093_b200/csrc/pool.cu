@@ -52,6 +52,7 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.score_part = take((rows + kScoreFoldRows - 1) / kScoreFoldRows * T * 8);
   l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
   l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
+  l.attn_cnt = take((size_t)kMaxTracesFast * c->num_kv_heads * 4);
   l.final_score = take(T * 4);
   l.answer = take(T * 4);
   l.finished = take(T);
@@ -82,6 +83,7 @@ __global__ void init_meta_kernel(DevViews v, Geo g, float unscored) {
     v.free_list[i] = g.num_blocks - 1 - (int)i;       // a stack: the first pop is block 0
   }
   for (size_t i = tid; i < (size_t)C_NUM; i += stride) v.counters[i] = (i == C_FREE_COUNT) ? g.num_blocks : 0;
+  for (size_t i = tid; i < (size_t)kMaxTracesFast * g.Hkv; i += stride) v.attn_cnt[i] = 0;
 }
 
 // ---------------------------------------------------------------- InitTraces (fork)
@@ -315,7 +317,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.prune_list = (int32_t*)(m + lay.prune_list); v.prune_off = (int32_t*)(m + lay.prune_off);
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
   v.score_part = (float2*)(m + lay.score_part);
-  v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o);
+  v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o); v.attn_cnt = (int32_t*)(m + lay.attn_cnt);
   v.final_score = (float*)(m + lay.final_score); v.answer = (int32_t*)(m + lay.answer);
   v.finished = (uint8_t*)(m + lay.finished); v.it_ids = (int32_t*)(m + lay.it_ids);
   v.it_fin = (int32_t*)(m + lay.it_fin); v.it_pruned = (int32_t*)(m + lay.it_pruned);

@@ -37,7 +37,7 @@ struct MetaLayout {
   size_t refcount, free_list, claim, counters;
   size_t append_base, prune_rank, prune_list, prune_off;
   size_t score_idx, score_z, score_part;
-  size_t attn_ml, attn_o;
+  size_t attn_ml, attn_o, attn_cnt;
   size_t final_score, answer, finished, it_ids, it_fin, it_pruned;
   size_t total;
 };
@@ -48,7 +48,7 @@ struct DevViews {
   int32_t* refcount; int32_t* free_list; int32_t* claim; int32_t* counters;
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
   int32_t* score_idx; float* score_z; float2* score_part;
-  float* attn_ml; float* attn_o;
+  float* attn_ml; float* attn_o; int32_t* attn_cnt;
   float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
   int32_t* it_ids; int32_t* it_fin; int32_t* it_pruned;       // per-iteration lists of the Algorithm 1 driver
 };
