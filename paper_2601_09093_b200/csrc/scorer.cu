@@ -5,7 +5,7 @@
 //
 // Only rows whose boundary flag is set are scored (Algorithm 1 runs the scorer when the new
 // token ends a step), so one launch is
-//   compact : ascending list of boundary rows (block-wide prefix sum), NaN into the other rows;
+//   compact : ascending list of boundary rows (prefix sums within and across the CTAs of a cluster), NaN into the other rows;
 //             it also decides, from the number of rows found, which first-layer kernel does the work
 //   mlp     : few rows (a decode step: about one boundary per 64 traces) - score_mlp_kernel, CUDA
 //             cores: for a tile of listed rows and a slice of the m hidden units the partial
@@ -17,6 +17,7 @@
 //             CTA partials in CTA order) and the mean is refreshed.
 #include "step_internal.cuh"
 
+#include <cooperative_groups.h>
 #include <math.h>
 
 using namespace stepk;
@@ -34,7 +35,7 @@ template <> __device__ inline float cvt<__nv_bfloat16>(__nv_bfloat16 x) { return
 
 // tc_min_rows: 0 = the tensor-core kernel is not available for this launch; otherwise the smallest
 // number of boundary rows that goes to it.  m: hidden units; num_sms: for the tiling choice.
-// One CTA; a thread looks at kRowsPerThread consecutive rows per pass.
+// A thread looks at kRowsPerThread consecutive rows per pass.
 // The step-end flag of row i is either mask[i] (tokens == nullptr) or, when the caller hands over the
 // sampled token ids instead, table[tokens[i]]: a token ends a step if its text contains "\n\n" (Sec. 3.1,
 // footnote), which the table records per vocabulary entry.  In that case the flags are also written to
@@ -55,51 +56,94 @@ __device__ inline bool row_flag(const FlagSource& f, int i, int32_t* counters) {
   return e;
 }
 
-__global__ void __launch_bounds__(kCompactThreads)
+// Block-wide exclusive prefix sum of one int per thread; *total gets the sum.
+__device__ inline int compact_scan(int x, int* s_warp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int w = s_warp[lane];
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    s_warp[lane] = wi - w;
+    if (lane == 31) s_warp[32] = wi;
+  }
+  __syncthreads();
+  *total = s_warp[32];
+  return s_warp[warp] + incl - x;
+}
+
+// A cluster of kCompactCtas CTAs; CTA r owns the r-th contiguous share of the rows.  Pass 1 counts the step-end
+// rows of the share, the counts are exchanged through distributed shared memory, pass 2 writes the row list
+// (ascending over the whole launch) and NaN into the other rows.
+constexpr int kCompactCtas = 8;
+
+__global__ void __cluster_dims__(kCompactCtas, 1, 1) __launch_bounds__(kCompactThreads, 1)
 score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step_scores,
                      int tc_min_rows, int m, int num_sms) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
   __shared__ int s_warp[33];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ int s_count, s_base, s_all;
   const float nan = __int_as_float(0x7fc00000);
-  int running = 0;
-  for (int base = 0; base < M; base += blockDim.x * kRowsPerThread) {
+  const int span = blockDim.x * kRowsPerThread;
+  const int share = ((M + C - 1) / C + span - 1) / span * span;       // rows per CTA, whole passes
+  const int lo = min(M, rank * share), hi = min(M, lo + share);
+  // pass 1: count
+  int mine = 0;
+  for (int base = lo; base < hi; base += span) {
+    const int i0 = base + threadIdx.x * kRowsPerThread;
+#pragma unroll
+    for (int j = 0; j < kRowsPerThread; ++j)
+      if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) ++mine;
+  }
+  {
+    int total;
+    compact_scan(mine, s_warp, &total);
+    if (threadIdx.x == 0) s_count = total;
+  }
+  cluster.sync();
+  if (threadIdx.x == 0) {
+    int before = 0, all = 0;
+    for (int r = 0; r < C; ++r) {
+      const int c = *cluster.map_shared_rank(&s_count, r);
+      if (r < rank) before += c;
+      all += c;
+    }
+    s_base = before; s_all = all;
+  }
+  __syncthreads();
+  // pass 2: place
+  int running = s_base;
+  for (int base = lo; base < hi; base += span) {
     const int i0 = base + threadIdx.x * kRowsPerThread;
     unsigned flags = 0;
 #pragma unroll
     for (int j = 0; j < kRowsPerThread; ++j)
-      if (i0 + j < M && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
-    const int mine = __popc(flags);
-    int incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int x = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += x;
-    }
-    __syncthreads();
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      const int w = s_warp[lane];
-      int wi = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int x = __shfl_up_sync(0xffffffffu, wi, o);
-        if (lane >= o) wi += x;
-      }
-      s_warp[lane] = wi - w;
-      if (lane == 31) s_warp[32] = wi;
-    }
-    __syncthreads();
-    int at = running + s_warp[warp] + incl - mine;
+      if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
+    int total;
+    int at = running + compact_scan(__popc(flags), s_warp, &total);
 #pragma unroll
     for (int j = 0; j < kRowsPerThread; ++j) {
       if (flags & (1u << j)) v.score_idx[at++] = i0 + j;
-      else if (i0 + j < M) step_scores[i0 + j] = nan;
+      else if (i0 + j < hi) step_scores[i0 + j] = nan;
     }
-    running += s_warp[32];
+    running += total;
   }
-  if (threadIdx.x == 0) {
-    const int nb = running;
+  if (rank == 0 && threadIdx.x == 0) {
+    const int nb = s_all;
     v.counters[C_SCORE_NB] = nb;
     v.counters[C_SCORE_TICKET] = 0;
     int N = 0;
@@ -116,6 +160,7 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
     v.counters[C_SCORE_TC] = N;
     v.counters[C_SCORE_SLICES] = N ? m / N : kSplits;
   }
+  cluster.sync();                        // no CTA leaves while its count may still be read
 }
 
 // grid (kSplits, row tiles).  Dynamic shared memory: kRowTile * D floats.
@@ -222,10 +267,16 @@ score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, in
   for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
     float sum = v.score_sum[t];
     int cnt = v.score_cnt[t];
-    for (int k = 0; k < chunks; ++k) {
-      const float2 p = __ldcg(&v.score_part[(size_t)k * g.max_traces + t]);
-      const int pc = __float_as_int(p.y);
-      if (pc) { sum += p.x; cnt += pc; }
+    for (int k0 = 0; k0 < chunks; k0 += 8) {
+      float2 p[8];                       // eight loads in flight, then added in CTA order
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        p[j] = k0 + j < chunks ? __ldcg(&v.score_part[(size_t)(k0 + j) * g.max_traces + t]) : make_float2(0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int pc = __float_as_int(p[j].y);
+        if (pc) { sum += p[j].x; cnt += pc; }
+      }
     }
     v.score_sum[t] = sum; v.score_cnt[t] = cnt;
     v.trace_scores[t] = cnt > 0 ? sum / (float)cnt : unscored;
@@ -314,7 +365,7 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
     if (part.tokens) part.tokens += off;
     if (part.mask_out) part.mask_out += off;
     if (part.live) part.live += off;
-    score_compact_kernel<<<1, kCompactThreads, 0, s>>>(pool->v, part, Mc, step_scores_out + off,
+    score_compact_kernel<<<kCompactCtas, kCompactThreads, 0, s>>>(pool->v, part, Mc, step_scores_out + off,
                                                        tc_min_rows, w->m, pool->num_sms);
     // the CUDA-core kernel only ever sees launches with fewer than tc_min_rows boundary rows
     const int scalar_rows = tc_min_rows > 0 && tc_min_rows - 1 < Mc ? tc_min_rows - 1 : Mc;

@@ -39,7 +39,6 @@ constexpr int kBoxRows = 64;                      // hidden units per TMA box
 constexpr int kBoxBytes = kBoxRows * kBK * 2;     // 8 KiB
 constexpr int kBBytes = kMaxN * kBK * 2;          // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
-constexpr int kLag = 3;                           // gather groups a producer thread keeps in flight
 constexpr int kEpiWarps = 4, kGatherWarps = 4;
 constexpr int kWarpTma = kEpiWarps + kGatherWarps, kWarpMma = kWarpTma + 1;
 constexpr int kThreads = (kWarpMma + 1) * 32;     // 320
@@ -95,10 +94,12 @@ __device__ inline bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned
 __device__ inline void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int kPending> __device__ inline void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+// The mbarrier gets one arrival from this thread once all its earlier cp.async copies have landed; the thread
+// itself does not wait.  (The barrier's expected count includes these arrivals: "noinc".)
+__device__ inline void cp_async_arrive_when_done(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ inline void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ inline void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -180,7 +181,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar_full + 8 * s, kGatherWarps + 1);            // one arrival per gather warp + the TMA thread
+      mbar_init(bar_full + 8 * s, kGatherWarps * 32 + 1);       // one arrival per gather thread + the TMA thread
       mbar_init(bar_empty + 8 * s, 1);                          // tcgen05.commit
     }
     for (int b = 0; b < 2; ++b) {
@@ -235,8 +236,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     const int tg = threadIdx.x - kEpiWarps * 32;                // 0 .. 127
     const int c = tg & 7, rb = tg >> 3;                         // 16-byte chunk of the row; rows rb + 16 i
     const uint32_t dst0 = base + (uint32_t)((rb >> 3) * 1024 + (rb & 7) * 128 + ((c ^ (rb & 7)) << 4));
-    const uint32_t my_full = bar_full;
-    int it = 0, signalled = 0;
+    int it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
       const int tile = item / slices;
@@ -255,23 +255,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) cp_async16(dst + i * 2048, src[i] + kr * kBK);
         if (++kr == KC) kr = 0;
-        cp_async_commit();
-        if (it >= kLag) {
-          cp_async_wait<kLag>();                                // chunk it - kLag of this thread has landed
-          fence_async_smem();                                   // ... and is visible to the tensor core's reads
-          __syncwarp();
-          if (lane == 0) mbar_arrive(my_full + 8 * ((it - kLag) % kStages));
-          ++signalled;
-        }
+        // the stage's barrier hears from this thread when these copies have landed; the thread moves on at once,
+        // so the copies of up to kStages chunks are in flight and nothing here waits for data
+        cp_async_arrive_when_done(bar_full + 8 * s);
       }
     }
-    cp_async_wait<0>();
-    fence_async_smem();
-    __syncwarp();
-    if (ok) {
-      for (; signalled < it; ++signalled)
-        if (lane == 0) mbar_arrive(my_full + 8 * (signalled % kStages));
-    } else {
+    cp_async_wait_all();                                        // nothing of this thread is in flight when it leaves
+    if (!ok) {
       if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
       *s_abort = 1;
     }
@@ -319,6 +309,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % kStages;
           if (*s_abort || !mbar_wait_bounded(bar_full + 8 * s, (it / kStages) & 1)) { ok = false; break; }
+          fence_async_smem();                                   // the gathered rows were written through the generic proxy
           tc_fence_after();
           const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes));
           const uint64_t bdesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + kABytes));
