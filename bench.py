@@ -164,7 +164,7 @@ def run_ours(args):
 
     K, Wm = args.steps, max(args.warmup, 3)
     e2e_steps = 0 if args.no_e2e else K
-    steps_total = Wm + K + (Wm + e2e_steps) + 4
+    steps_total = Wm + K + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS + 3
     free_b, total_b = torch.cuda.mem_get_info(dev)
     cfg, suffix, nb, max_pages, phys_layers = workload_plan(args.workload, args.num_blocks, steps_total, free_b)
     cfg_pool = W.scaled(cfg, num_layers=phys_layers)
@@ -318,6 +318,7 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         res["cpu_baseline"], res["sampled_parity"] = cpu_baseline_and_parity(pool, cfg, sets[(K - 1) % NSETS], out, L, phys_layers)
     if not args.no_aux:
+        res["algorithm1_loop"] = algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host, ms_total / K)
         res["scorer"] = scorer_measurements(cfg, dev, rows=args.scorer_rows)
         if args.workload == "c3":
             # last: this consumes the benchmark state (the pool ends with two live traces)
@@ -382,6 +383,66 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
 
 
 # ---------------------------------------------------------------------------------------------
+ALG1_ITERATIONS = 6
+
+
+def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host, ms_per_step_python):
+    """The same decode step driven by the library's own loop (algorithm1_run: one C call for all iterations, step-end
+    flags taken from sampled token ids, completion handling included) instead of one Python call per kernel group.
+    No trace samples the end-of-sequence token and the trigger stays quiet, so the work per iteration equals a step
+    of the timed region.  Also times detect_step_ends alone on 4M tokens."""
+    import torch
+    from paper_2601_09093_b200 import binding as B, workloads as W
+    vocab = W.synthetic_vocab(cfg.seed, 32000, step_end_frac=0.01)
+    table = B.step_end_table_from_vocab(vocab)
+    ends = np.flatnonzero(table.numpy())
+    toks = np.stack([W.token_ids(cfg.seed, T, len(vocab), ends, cfg.boundary_density, sub=500 + i)
+                     for i in range(ALG1_ITERATIONS + 2)])
+    toks[toks == 0] = 1                                            # id 0 is the end-of-sequence token here: nobody completes
+    table_d, toks_d = table.to(dev), torch.from_numpy(toks).to(dev)
+    q = torch.stack([s["q"][:phys_layers] for s in sets]).contiguous()
+    k = torch.stack([s["k"] for s in sets]).contiguous()
+    v = torch.stack([s["v"] for s in sets]).contiguous()
+    h = torch.stack([s["h"] for s in sets]).contiguous()
+    answers = torch.zeros(T, dtype=torch.int32, device=dev)
+    attn_out = torch.empty((phys_layers, T, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
+
+    def run(tok, n):
+        r = pool.algorithm1_run(tok, 0, table_d, answers, q, k, v, h, wts, cfg.threshold, cfg.keep_frac,
+                                check_every=n, attn_out=attn_out)
+        for _ in range(n):
+            append_log.append((ids_host, 1))
+        return r
+
+    run(toks_d[:2], 2)                                              # warm-up
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    r = run(toks_d[2:], ALG1_ITERATIONS)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / ALG1_ITERATIONS
+    # step-end detection alone
+    n_tok = 1 << 22
+    big = torch.from_numpy(W.token_ids(cfg.seed, n_tok, len(vocab), ends, cfg.boundary_density, sub=77)).to(dev)
+    mask = torch.empty(n_tok, dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        pool.detect_step_ends(big, table_d, mask)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(11)]
+    ev[0].record()
+    for i in range(10):
+        pool.detect_step_ends(big, table_d, mask)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    det_ms = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(10)]))
+    code, bits = pool.last_error()
+    return {"iterations": r["iterations"], "ms_per_iteration": ms, "trace_decode_steps_per_s": T / (ms * 1e-3),
+            "vs_python_driven_step": ms_per_step_python / ms, "launches_per_iteration": 8 + phys_layers,
+            "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
+            "detect_step_ends": {"tokens": n_tok, "us_per_call": det_ms * 1e3, "tokens_per_s": n_tok / (det_ms * 1e-3),
+                                 "gbs": n_tok * 5 / (det_ms * 1e-3) / 1e9},
+            "device_error_mask": bits}
+
+
 def scorer_measurements(cfg, dev, rows=65536, reps=20, all_rows_density=1.0):
     """score_steps timed alone (CUDA events around each call, median of `reps`) on three shapes of one scorer:
     a decode step (one row per trace, Bernoulli step-end flags), the batched shape (1024 rows per trace at the
