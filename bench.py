@@ -51,10 +51,10 @@ def parse_args():
 
 
 # DRAM bytes moved per algorithmic byte by attn_mma_kernel: dram__bytes_read.sum + dram__bytes_write.sum of one
-# ncu capture on the one-layer 64-trace workload (2.6895 GB + 6.56 MB against 2.665 GB algorithmic; the summary is
+# ncu capture on the one-layer 64-trace workload (2.6920 GB + 6.64 MB against 2.6628 GB algorithmic; the summary is
 # profiles/attn_mma_kernel_C1_ncu_full.md).  The kernel streams every page once, so traffic grows in proportion to
 # the algorithmic bytes and the larger workloads scale this figure.  Set to None when the kernel changes.
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (2.6895e9 + 6.56e6) / 2.665e9
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (2.692034e9 + 6.6432e6) / 2.662836852e9
 
 
 def measured_peaks(key="hbm_gbs", fallback=6650.0):
@@ -318,7 +318,8 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         res["cpu_baseline"], res["sampled_parity"] = cpu_baseline_and_parity(pool, cfg, sets[(K - 1) % NSETS], out, L, phys_layers)
     if not args.no_aux:
-        res["algorithm1_loop"] = algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host, ms_total / K)
+        res["algorithm1_loop"] = algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host,
+                                                        ms_total / K if phys_layers == L else None)
         res["scorer"] = scorer_measurements(cfg, dev, rows=args.scorer_rows)
         if args.workload == "c3":
             # last: this consumes the benchmark state (the pool ends with two live traces)
@@ -436,7 +437,8 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     det_ms = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(10)]))
     code, bits = pool.last_error()
     return {"iterations": r["iterations"], "ms_per_iteration": ms, "trace_decode_steps_per_s": T / (ms * 1e-3),
-            "vs_python_driven_step": ms_per_step_python / ms, "launches_per_iteration": 8 + phys_layers,
+            "vs_python_driven_step": None if ms_per_step_python is None else ms_per_step_python / ms,
+            "layers_per_iteration": phys_layers, "launches_per_iteration": 8 + phys_layers,
             "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
             "detect_step_ends": {"tokens": n_tok, "us_per_call": det_ms * 1e3, "tokens_per_s": n_tok / (det_ms * 1e-3),
                                  "gbs": n_tok * 5 / (det_ms * 1e-3) / 1e9},

@@ -101,13 +101,17 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
   const int span = blockDim.x * kRowsPerThread;
   const int share = ((M + C - 1) / C + span - 1) / span * span;       // rows per CTA, whole passes
   const int lo = min(M, rank * share), hi = min(M, lo + share);
-  // pass 1: count
+  // pass 1: count (the flags of the share's first pass stay in a register for pass 2)
   int mine = 0;
+  unsigned first_flags = 0;
   for (int base = lo; base < hi; base += span) {
     const int i0 = base + threadIdx.x * kRowsPerThread;
+    unsigned flags = 0;
 #pragma unroll
     for (int j = 0; j < kRowsPerThread; ++j)
-      if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) ++mine;
+      if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
+    if (base == lo) first_flags = flags;
+    mine += __popc(flags);
   }
   {
     int total;
@@ -129,10 +133,13 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
   int running = s_base;
   for (int base = lo; base < hi; base += span) {
     const int i0 = base + threadIdx.x * kRowsPerThread;
-    unsigned flags = 0;
+    unsigned flags = first_flags;
+    if (base != lo) {
+      flags = 0;
 #pragma unroll
-    for (int j = 0; j < kRowsPerThread; ++j)
-      if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
+      for (int j = 0; j < kRowsPerThread; ++j)
+        if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
+    }
     int total;
     int at = running + compact_scan(__popc(flags), s_warp, &total);
 #pragma unroll
