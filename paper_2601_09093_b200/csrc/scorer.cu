@@ -28,6 +28,7 @@ constexpr int kCompactThreads = 1024;
 constexpr int kRowTile = 8;       // listed rows per CTA
 constexpr int kSplits = kScoreSplits;   // slices of the m hidden units
 constexpr int kMlpWarps = 4;
+constexpr int kFinishThreads = 1024;
 
 template <typename T> __device__ inline float cvt(T x);
 template <> __device__ inline float cvt<float>(float x) { return x; }
@@ -163,6 +164,8 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
         N = cand;
         if (tiles * (m / cand) >= num_sms) break;
       }
+      // items of 256 rows (two accumulators sharing each W1 tile) if there are still enough of them
+      v.counters[C_SCORE_TILE] = ((nb + 255) / 256) * (m / N) >= num_sms ? 256 : 128;
     }
     v.counters[C_SCORE_TC] = N;
     v.counters[C_SCORE_SLICES] = N ? m / N : kSplits;
@@ -234,11 +237,12 @@ score_mlp_kernel(DevViews v, const T* __restrict__ hidden, const T* __restrict__
 //      (a thread per trace walks the CTA's rows in shared memory), written as one partial;
 //   3. the CTA that finishes last adds the partials of every trace in CTA order to the trace's running
 //      (sum, count) and refreshes the mean - a fixed order, whichever CTA happens to be last.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kFinishThreads)
 score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, int row_base, float b2,
                     float unscored, float* __restrict__ step_scores) {
   __shared__ float s_y[kScoreFoldRows];
   __shared__ int s_tr[kScoreFoldRows];
+  __shared__ float2 s_run[kFinishThreads];
   __shared__ int s_last;
   const int nb = v.counters[C_SCORE_NB], ns = v.counters[C_SCORE_SLICES];
   const int chunks = (nb + kScoreFoldRows - 1) / kScoreFoldRows;
@@ -271,22 +275,44 @@ score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, in
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
-    float sum = v.score_sum[t];
-    int cnt = v.score_cnt[t];
-    for (int k0 = 0; k0 < chunks; k0 += 8) {
-      float2 p[8];                       // eight loads in flight, then added in CTA order
+  // every trace's partials are summed by `groups` threads, each over a contiguous run of CTAs, and the runs are
+  // then added in order: the same fixed order whoever is last, with the loads spread over the whole CTA
+  const int T = g.max_traces;
+  const int Tc = min(T, (int)blockDim.x), groups = max(1, (int)blockDim.x / Tc);
+  const int cpg = (chunks + groups - 1) / groups;
+  const int tl = threadIdx.x % Tc, grp = threadIdx.x / Tc;
+  for (int base = 0; base < T; base += Tc) {
+    const int t = base + tl;
+    float sum = 0.f;
+    int cnt = 0;
+    if (grp < groups && t < T) {
+      const int k_end = min(chunks, (grp + 1) * cpg);
+      for (int k0 = grp * cpg; k0 < k_end; k0 += 8) {
+        float2 p[8];                       // eight loads in flight, then added in CTA order
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
-        p[j] = k0 + j < chunks ? __ldcg(&v.score_part[(size_t)(k0 + j) * g.max_traces + t]) : make_float2(0.f, 0.f);
+        for (int j = 0; j < 8; ++j)
+          p[j] = k0 + j < k_end ? __ldcg(&v.score_part[(size_t)(k0 + j) * T + t]) : make_float2(0.f, 0.f);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int pc = __float_as_int(p[j].y);
-        if (pc) { sum += p[j].x; cnt += pc; }
+        for (int j = 0; j < 8; ++j) {
+          const int pc = __float_as_int(p[j].y);
+          if (pc) { sum += p[j].x; cnt += pc; }
+        }
       }
     }
-    v.score_sum[t] = sum; v.score_cnt[t] = cnt;
-    v.trace_scores[t] = cnt > 0 ? sum / (float)cnt : unscored;
+    s_run[threadIdx.x] = make_float2(sum, __int_as_float(cnt));
+    __syncthreads();
+    if (grp == 0 && t < T) {
+      float tot = v.score_sum[t];
+      int n_tot = v.score_cnt[t];
+      for (int q = 0; q < groups; ++q) {
+        const float2 r = s_run[q * Tc + tl];
+        const int rc = __float_as_int(r.y);
+        if (rc) { tot += r.x; n_tot += rc; }
+      }
+      v.score_sum[t] = tot; v.score_cnt[t] = n_tot;
+      v.trace_scores[t] = n_tot > 0 ? tot / (float)n_tot : unscored;
+    }
+    __syncthreads();
   }
 }
 
@@ -395,7 +421,7 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
       if (st != STEP_OK) return st;
     }
     // row_trace == NULL means row i is trace i, counted from the start of the whole call
-    score_finish_kernel<<<(Mc + kScoreFoldRows - 1) / kScoreFoldRows, 256, 0, s>>>(
+    score_finish_kernel<<<(Mc + kScoreFoldRows - 1) / kScoreFoldRows, kFinishThreads, 0, s>>>(
         pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off);
   }
   return launch_ok();

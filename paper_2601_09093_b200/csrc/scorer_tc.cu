@@ -1,21 +1,22 @@
 // Tensor-core form of the step scorer's first layer for launches with many boundary rows
 // (Sec. 3.1 "Model Architecture": y = sigmoid(w2 . ReLU(W1 h + b1) + b2)).
 //
-// For the listed rows r and a slice [n0, n0 + N) of the m hidden units one work item computes
+// For up to 256 listed rows r (two halves of 128; launches too small to fill the SMs that way use 128) and a slice [n0, n0 + N) of the m hidden units one work item computes
 //     z_slice[r] = sum_{j in slice} w2[j] * ReLU(sum_k h[r][k] * W1[j][k] + b1[j])
-// as a 128 x N x D bf16 GEMM on the 5th-generation tensor cores with the whole second layer fused into
-// the read-out of the accumulator:
-//   * the accumulator (128 rows x N columns, fp32) lives in tensor memory; two of them (2 x 256 columns)
-//     let the read-out of one item overlap the products of the next;
+// as a 256 x N x D bf16 GEMM on the 5th-generation tensor cores with the whole second layer fused into
+// the read-out of the accumulators:
+//   * two accumulators (128 rows x N columns each, fp32) live in tensor memory (2 x 256 columns); both row
+//     halves multiply the same W1 tile, which halves the W1 bytes fetched per product - operand delivery from
+//     L2, not the tensor pipe, is what limits this kernel;
 //   * A = the hidden rows named by the row list.  The rows are scattered in the caller's [M, D]
-//     array, so four warps gather them with 16-byte cp.async copies straight into the 128-byte-swizzled
+//     array, so eight warps gather them with 16-byte cp.async copies straight into the 128-byte-swizzled
 //     K-major arrangement the MMA unit reads (row r of a tile at (r / 8) * 1024 + (r % 8) * 128,
 //     16-byte chunk c stored at chunk c ^ (r % 8)); no compacted copy of the rows is ever made;
 //   * B = W1[n0 .. n0 + N, k .. k + 64): TMA tiled loads (one 64 x 64 box per 64 units, 128-byte
 //     swizzle) signalling the stage's mbarrier with their byte count;
-//   * one thread issues tcgen05.mma (M 128, N 64 | 128 | 256, K 16) four times per 64-wide k-chunk and
+//   * one thread issues tcgen05.mma (M 128, N 64 | 128 | 256, K 16) four times per row half and 64-wide k-chunk and
 //     commits the stage back to the producers;
-//   * four warps read the finished accumulator with tcgen05.ld - a thread owns one row, so
+//   * eight warps read the finished accumulators with tcgen05.ld - a thread owns one row, so
 //     + b1, ReLU, * w2 and the sum over the slice's units are plain per-thread fp32 arithmetic on
 //     un-rounded activations - and store one partial per (row, slice) for the finishing kernel.
 // The kernel is persistent (one CTA per SM, items handed out round-robin).  N is picked on the device
@@ -30,19 +31,20 @@ using namespace stepk;
 
 namespace {
 
-constexpr int kTileRows = 128;                    // UMMA M: rows of one item
+constexpr int kHalfRows = 128;                    // UMMA M
 constexpr int kBK = 64;                           // bf16 elements per k-chunk (one 128-byte swizzle row)
 constexpr int kMaxN = 256;                        // UMMA N limit
-constexpr int kStages = 4;
-constexpr int kABytes = kTileRows * kBK * 2;      // 16 KiB
+constexpr int kStages = 3;
+constexpr int kHalfBytes = kHalfRows * kBK * 2;   // 16 KiB
+constexpr int kABytes = 2 * kHalfBytes;           // 32 KiB
 constexpr int kBoxRows = 64;                      // hidden units per TMA box
 constexpr int kBoxBytes = kBoxRows * kBK * 2;     // 8 KiB
 constexpr int kBBytes = kMaxN * kBK * 2;          // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;    // 48 KiB
-constexpr int kEpiWarps = 4, kGatherWarps = 4;
+constexpr int kStageBytes = kABytes + kBBytes;    // 64 KiB
+constexpr int kEpiWarps = 8, kGatherWarps = 8;    // read-out: warp w takes TMEM lanes 32 (w % 4) of accumulator w / 4
 constexpr int kWarpTma = kEpiWarps + kGatherWarps, kWarpMma = kWarpTma + 1;
-constexpr int kThreads = (kWarpMma + 1) * 32;     // 320
-constexpr int kTmemCols = 512;                    // two accumulators of up to 256 columns
+constexpr int kThreads = (kWarpMma + 1) * 32;     // 576
+constexpr int kTmemCols = 512;                    // two accumulators (row halves) of up to 256 columns
 constexpr int kMaxUnits = 1024;                   // b1 / w2 staged in shared memory as fp32
 constexpr unsigned long long kWaitNs = 2000000000ull;
 constexpr unsigned long long kDrainNs = 100000000ull;
@@ -151,7 +153,7 @@ __device__ inline int first_chunk(int item, int KC) { return (int)(((unsigned)it
 
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
 __device__ inline uint32_t umma_idesc_bf16(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kHalfRows >> 4) << 24);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -161,7 +163,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   if (N == 0) return;
   const int nb = a.counters[C_SCORE_NB];
   const int slices = a.m / N;
-  const int tiles = (nb + kTileRows - 1) / kTileRows;
+  const int R = a.counters[C_SCORE_TILE];                       // rows per item: 256, or 128 for launches too small to
+  const int tiles = (nb + R - 1) / R;                           // fill the SMs with 256-row items
   const int items = tiles * slices;
   const int KC = a.D / kBK;
 
@@ -172,10 +175,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   float* s_b1 = reinterpret_cast<float*>(sm + kStages * kStageBytes);
   float* s_w2 = s_b1 + kMaxUnits;
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_w2 + kMaxUnits);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 4);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 2);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const uint32_t bar_full = smem_u32(s_bar), bar_empty = bar_full + 8 * kStages;
-  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 16;
+  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 8;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -184,10 +187,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       mbar_init(bar_full + 8 * s, kGatherWarps * 32 + 1);       // one arrival per gather thread + the TMA thread
       mbar_init(bar_empty + 8 * s, 1);                          // tcgen05.commit
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(bar_tfull + 8 * b, 1);                          // tcgen05.commit
-      mbar_init(bar_tempty + 8 * b, kEpiWarps);                 // one arrival per read-out warp
-    }
+    mbar_init(bar_tfull, 1);                                    // tcgen05.commit
+    mbar_init(bar_tempty, kEpiWarps);                           // one arrival per read-out warp
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -205,36 +206,39 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   const uint32_t tmem_base = *s_tmem;
 
   if (warp < kEpiWarps) {
-    // ------------------------------------------------ read-out: second layer on the accumulator
+    // ------------------------------------------------ read-out: second layer on the accumulators
+    const int quarter = warp & 3, half = warp >> 2;
     int li = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, ++li) {
       const int tile = item / slices, slice = item - tile * slices, n0 = slice * N;
-      const int buf = li & 1;
       if (*s_abort) break;
-      if (!mbar_wait_bounded(bar_tfull + 8 * buf, (li >> 1) & 1)) {
+      if (!mbar_wait_bounded(bar_tfull, li & 1)) {
         if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
         *s_abort = 1;
         break;
       }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kMaxN);
+      const int row = tile * R + half * kHalfRows + quarter * 32 + lane;
+      const bool used = half * kHalfRows < R && tile * R + half * kHalfRows < nb;   // did this half get any products?
       float z = 0.f;
-      for (int c0 = 0; c0 < N; c0 += 32) {
-        float v[32];
-        tc_ld32(taddr + c0, v);
+      if (used) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kMaxN);
+        for (int c0 = 0; c0 < N; c0 += 32) {
+          float v[32];
+          tc_ld32(taddr + c0, v);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) z = fmaf(s_w2[n0 + c0 + j], fmaxf(v[j] + s_b1[n0 + c0 + j], 0.f), z);
+          for (int j = 0; j < 32; ++j) z = fmaf(s_w2[n0 + c0 + j], fmaxf(v[j] + s_b1[n0 + c0 + j], 0.f), z);
+        }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-      const int row = tile * kTileRows + warp * 32 + lane;
-      if (row < nb) a.z[(size_t)row * kScoreSplits + slice] = z;
+      if (lane == 0) mbar_arrive(bar_tempty);
+      if (used && row < nb) a.z[(size_t)row * kScoreSplits + slice] = z;
     }
   } else if (warp < kWarpTma) {
     // ------------------------------------------------ gather of the listed hidden rows into A
-    const int tg = threadIdx.x - kEpiWarps * 32;                // 0 .. 127
-    const int c = tg & 7, rb = tg >> 3;                         // 16-byte chunk of the row; rows rb + 16 i
+    const int tg = threadIdx.x - kEpiWarps * 32;                // 0 .. 255
+    const int c = tg & 7, rb = tg >> 3;                         // 16-byte chunk of the row; rows rb + 32 i
     const uint32_t dst0 = base + (uint32_t)((rb >> 3) * 1024 + (rb & 7) * 128 + ((c ^ (rb & 7)) << 4));
     int it = 0;
     bool ok = true;
@@ -243,17 +247,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       const __nv_bfloat16* src[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        int gr = tile * kTileRows + rb + 16 * i;
+        int gr = tile * R + rb + 32 * i;
         if (gr >= nb) gr = nb - 1;                              // rows past the list re-read its last row; never stored
         src[i] = a.hidden + (size_t)a.idx[gr] * a.D + c * 8;
       }
+      const int n_copy = R > kHalfRows && tile * R + kHalfRows < nb ? 8 : 4;   // the second half may be absent or empty
       int kr = first_chunk(item, KC);
       for (int kc = 0; kc < KC; ++kc, ++it) {
         const int s = it % kStages;
         if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
         const uint32_t dst = dst0 + (uint32_t)(s * kStageBytes);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16(dst + i * 2048, src[i] + kr * kBK);
+        for (int i = 0; i < 8; ++i)
+          if (i < n_copy) cp_async16(dst + i * 4096, src[i] + kr * kBK);
         if (++kr == KC) kr = 0;
         // the stage's barrier hears from this thread when these copies have landed; the thread moves on at once,
         // so the copies of up to kStages chunks are in flight and nothing here waits for data
@@ -302,23 +308,27 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       int it = 0, li = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++li) {
-        const int buf = li & 1;
-        if (*s_abort || !mbar_wait_bounded(bar_tempty + 8 * buf, ((li >> 1) & 1) ^ 1)) { ok = false; break; }
+        const int tile = item / slices;
+        const int halves = R > kHalfRows && tile * R + kHalfRows < nb ? 2 : 1;
+        // the read-out of the previous item must have drained the accumulators
+        if (*s_abort || !mbar_wait_bounded(bar_tempty, (li & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kMaxN);
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % kStages;
           if (*s_abort || !mbar_wait_bounded(bar_full + 8 * s, (it / kStages) & 1)) { ok = false; break; }
           fence_async_smem();                                   // the gathered rows were written through the generic proxy
           tc_fence_after();
-          const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes));
           const uint64_t bdesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + kABytes));
+          for (int h = 0; h < halves; ++h) {                    // both row halves multiply the same W1 tile
+            const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + h * kHalfBytes));
+            const uint32_t d_tmem = tmem_base + (uint32_t)(h * kMaxN);
 #pragma unroll
-          for (int kk = 0; kk < kBK / 16; ++kk)                  // 16 bf16 = 32 bytes further along the swizzled row
-            tc_mma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | kk) != 0);
+            for (int kk = 0; kk < kBK / 16; ++kk)                // 16 bf16 = 32 bytes further along the swizzled row
+              tc_mma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | kk) != 0);
+          }
           tc_commit(bar_empty + 8 * s);                         // the stage is free once these products have read it
         }
-        if (ok) tc_commit(bar_tfull + 8 * buf);                 // the accumulator is complete
+        if (ok) tc_commit(bar_tfull);                           // the accumulators are complete
       }
       if (!ok) {
         flag_error(a.counters, STEP_ERR_TIMEOUT);
@@ -337,7 +347,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
 }
 
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 2 * kMaxUnits * sizeof(float) +
-                              (2 * kStages + 4) * sizeof(uint64_t) + 16;
+                              (2 * kStages + 2) * sizeof(uint64_t) + 16;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -389,7 +399,7 @@ int score_tc_launch(const step_pool* pool, const void* hidden, int Mc, const sco
   a.b1 = (const __nv_bfloat16*)w->b1; a.w2 = (const __nv_bfloat16*)w->w2;
   a.idx = pool->v.score_idx; a.z = pool->v.score_z; a.counters = pool->v.counters;
   a.D = w->D; a.m = w->m;
-  long long max_items = (long long)((Mc + kTileRows - 1) / kTileRows) * (w->m / kBoxRows);
+  long long max_items = (long long)((Mc + kHalfRows - 1) / kHalfRows) * (w->m / kBoxRows);
   int grid = pool->num_sms;
   if (max_items < grid) grid = (int)max_items;
   if (grid < 1) grid = 1;

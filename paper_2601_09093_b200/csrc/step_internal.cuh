@@ -30,7 +30,9 @@ constexpr int kScoreFoldRows = 512;    // listed rows one CTA of the scorer's fi
 enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_PRUNE_N = 4,
                C_SCORE_TC = 5, C_SCORE_SLICES = 6, C_SCORE_TICKET = 7,
                // Algorithm 1 driver: live / finishing traces of the current iteration, running totals
-               C_IT_NLIVE = 8, C_IT_NFIN = 9, C_N_FINISHED = 10, C_N_EVICTED = 11, C_IT_NPRUNED = 12, C_NUM = 64 };
+               C_IT_NLIVE = 8, C_IT_NFIN = 9, C_N_FINISHED = 10, C_N_EVICTED = 11, C_IT_NPRUNED = 12,
+               C_SCORE_TILE = 13,   // rows per work item of the tensor-core scorer kernel (128 or 256)
+               C_NUM = 64 };
 
 struct MetaLayout {
   size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;

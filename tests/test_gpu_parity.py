@@ -314,7 +314,7 @@ def test_scorer_picks_the_cuda_core_kernel_below_the_row_threshold():
     _scorer_case(W.C1, 512, 1.0, row_trace=rt, max_score_rows=512, mode=-1, expect_tc=0)    # forced off
 
 
-@pytest.mark.parametrize("rows,units", [(4800, 128), (9600, 256)])
+@pytest.mark.parametrize("rows,units", [(4800, 128), (9600, 256), (19000, 256)])
 def test_scorer_tensor_core_wide_slices_sampled(rows, units):
     """Launches large enough that the device picks 128- and 256-unit slices (several items per CTA, both
     accumulators in use).  The oracle scores a sample of rows; the CUDA-core kernel, itself checked against
