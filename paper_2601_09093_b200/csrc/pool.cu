@@ -382,7 +382,7 @@ int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int 
   Geo g = geo_of(pool);
   const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
   const size_t row_chunks = (size_t)n_tokens * g.L * g.Hkv * cpr;   // 16-byte chunks of K (or V) per trace
-  constexpr int kListChunk = 4096;                                  // traces per launch (shared-memory scan)
+  constexpr int kListChunk = 2048;                                  // traces per launch (24 KiB of shared memory for the scan)
   for (int off = 0; off < n; off += kListChunk) {
     const int m = n - off < kListChunk ? n - off : kListChunk;
     if (n_dev && off > 0) return STEP_ERR_INVALID_ARG;              // a device-side count covers one launch only

@@ -1,0 +1,107 @@
+"""GPU parity at the edges of what the kernels are built for: largest trace counts of the fast paths and the
+fallbacks just beyond them, full block tables, lists longer than the shared-memory staging, the paper's third
+scorer width."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as OA
+from oracle import scorer as OS
+from paper_2601_09093_b200 import binding as B
+from paper_2601_09093_b200 import harness as H
+from paper_2601_09093_b200 import workloads as W
+
+from gpu_common import Twin, exact_f32, attention_errors
+
+pytestmark = pytest.mark.gpu
+
+
+def _many_short_traces(n, seed):
+    """n traces sharing a 16-token prompt, 0-40 further tokens each (some stay at the bare prompt)."""
+    cfg = W.scaled(W.C1, n_traces=n, num_q_heads=8, num_kv_heads=2, prefix_len=16, seed=seed)
+    tw = Twin(cfg, n * 3 + 8, 4, n)
+    ids, _ = tw.fork(n, 16)
+    extra = W.rng(seed, W.TID_LEN).integers(0, 41, size=n)
+    for sel, inc in H.ragged_append_plan(extra):
+        assert all(tw.append([ids[i] for i in sel], inc))
+    return cfg, tw
+
+
+@pytest.mark.parametrize("n", [2048, 2049])
+def test_attention_at_and_beyond_the_tensor_core_kernels_trace_limit(n):
+    """2048 rows is the most the tensor-core kernel takes in one call; 2049 goes to the scalar kernel."""
+    cfg, tw = _many_short_traces(n, 31)
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (n, 8, 128), "bf16")
+    v = tw.gpu.views()
+    got = exact_f32(tw.gpu.decode_attention(0, H.to_device(qb, "bf16"), v["block_table"], v["seq_lens"]))
+    want = OA.paged_decode_attention(qx, tw.ora.k_pages[0], tw.ora.v_pages[0], tw.ora.block_table, tw.ora.seq_lens)
+    mx, mean = attention_errors(got, want)
+    assert mx <= 1e-2 and mean <= 1e-3
+    assert tw.status() == (0, 0)
+
+
+def test_full_block_table_and_capacity_errors():
+    """A trace that fills its block table to the last slot attends over all of it; one more token is refused."""
+    cfg = W.scaled(W.C1, n_traces=2, num_q_heads=8, num_kv_heads=2, prefix_len=16)
+    tw = Twin(cfg, 24, 8, 2)                                     # 8 pages = 128 tokens per trace at most
+    ids, _ = tw.fork(2, 16)
+    assert all(tw.append(ids, 112))
+    assert tw.append(ids[:1], 1) == [False]                       # table full: skipped and flagged on both sides
+    mask, omask = tw.status()
+    assert mask == omask == 1 << 4
+    tw.assert_meta_equal()
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (2, 8, 128), "bf16")
+    v = tw.gpu.views()
+    got = exact_f32(tw.gpu.decode_attention(0, H.to_device(qb, "bf16"), v["block_table"], v["seq_lens"]))
+    want = OA.paged_decode_attention(qx, tw.ora.k_pages[0], tw.ora.v_pages[0], tw.ora.block_table, tw.ora.seq_lens)
+    mx, mean = attention_errors(got, want)
+    assert mx <= 1e-2 and mean <= 1e-3
+
+
+def test_prune_list_longer_than_the_shared_memory_staging():
+    """2048 live traces, three quarters evicted: the eviction list (1536) exceeds what the release stages in shared
+    memory, so the offsets come from global memory; free list and tables must still match the oracle bit for bit."""
+    n = 2048
+    cfg = W.scaled(W.C0, n_traces=n, prefix_len=16)
+    tw = Twin(cfg, n * 3 + 8, 4, n, store_payload=False)
+    ids, _ = tw.fork(n, 16)
+    extra = W.rng(7, W.TID_LEN).integers(1, 33, size=n)
+    for sel, inc in H.ragged_append_plan(extra):
+        assert all(tw.append([ids[i] for i in sel], inc))
+    scores = W.rng(7, W.TID_ANS).random(n).astype(np.float32)
+    scores[::97] = scores[5]                                       # ties
+    pid, npr = tw.gpu.prune_if_saturated(torch.from_numpy(scores).cuda(), 0.01, 0.25)
+    got = pid[: int(npr.item())].cpu().tolist()
+    assert got == tw.ora.prune_if_saturated(scores, 0.01, 0.25) and len(got) == 1536
+    tw.assert_meta_equal()
+    assert tw.status() == (0, 0)
+
+
+def test_append_list_longer_than_one_launch():
+    """5000 traces in one append_kv call: the list is served in several launches, in list order."""
+    n = 5000
+    cfg = W.scaled(W.C0, n_traces=n, prefix_len=16)
+    tw = Twin(cfg, n + 64, 3, n, store_payload=False)
+    ids, _ = tw.fork(n, 16)
+    order = W.rng(3, W.TID_PERM).permutation(n).tolist()          # not ascending: allocation follows the list
+    assert all(tw.append(order, 1))
+    tw.assert_meta_equal()
+    assert tw.status() == (0, 0)
+
+
+def test_scorer_width_2560_on_the_tensor_cores():
+    """The paper's smallest hidden size (2560, scorer width 512): 40 k-chunks, a count that is not a power of two."""
+    cfg = W.scaled(W.C1, scorer_D=2560, scorer_m=512)
+    M, T = 700, 64
+    pool = H.make_pool(cfg, 8, 4, T, max_score_rows=M)
+    (W1b, W1x), (b1b, b1x), (w2b, w2x), b2 = W.scorer_weights(cfg, bias_std=0.05)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16"), H.to_device(b1b, "bf16"), H.to_device(w2b, "bf16"), b2, B.STEP_BF16)
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (M, 2560), "bf16")
+    mask = W.boundary_mask(cfg, M, density=0.5)
+    rt = torch.from_numpy((np.arange(M) % T).astype(np.int32)).cuda()
+    got = pool.score_steps(H.to_device(hb, "bf16"), torch.from_numpy(mask).cuda(), rt, wts).cpu().numpy()
+    assert pool.score_launch_info()["tc_units"] == 64
+    want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+    assert np.abs(got[mask == 1] - want[mask == 1]).max() <= 1e-3
+    assert OS.scorer_flops(512, 2560) == 2622464                  # the appendix's 2m(d+1)
+    assert pool.last_error() == (0, 0)
