@@ -383,7 +383,6 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
   if (!w->W1 || !w->b1 || !w->w2 || w->D < 1 || w->m < 1) return STEP_ERR_INVALID_ARG;
   if (w->dtype != STEP_BF16 && w->dtype != STEP_FP32) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)kRowTile * w->D * sizeof(float);
-  if (smem > 200 * 1024) return STEP_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   Geo g = geo_of(pool);
   const size_t eb = w->dtype == STEP_BF16 ? 2 : 4;
@@ -403,6 +402,7 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
     // the CUDA-core kernel only ever sees launches with fewer than tc_min_rows boundary rows
     const int scalar_rows = tc_min_rows > 0 && tc_min_rows - 1 < Mc ? tc_min_rows - 1 : Mc;
     if (scalar_rows > 0) {
+      if (smem > 200 * 1024) return STEP_ERR_INVALID_ARG;           // the CUDA-core kernel stages 8 hidden rows as fp32
       dim3 grid(kSplits, (scalar_rows + kRowTile - 1) / kRowTile);
       if (w->dtype == STEP_BF16) {
         auto kern = score_mlp_kernel<__nv_bfloat16>;

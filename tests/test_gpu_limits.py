@@ -105,3 +105,22 @@ def test_scorer_width_2560_on_the_tensor_cores():
     assert np.abs(got[mask == 1] - want[mask == 1]).max() <= 1e-3
     assert OS.scorer_flops(512, 2560) == 2622464                  # the appendix's 2m(d+1)
     assert pool.last_error() == (0, 0)
+
+
+def test_scorer_width_8192_runs_on_the_tensor_cores_only():
+    """D = 8192 is more than the CUDA-core kernel can stage; the tensor-core kernel takes it, the other path says no."""
+    cfg = W.scaled(W.C1, scorer_D=8192, scorer_m=256)
+    M, T = 300, 64
+    pool = H.make_pool(cfg, 8, 4, T, max_score_rows=M)
+    (W1b, W1x), (b1b, b1x), (w2b, w2x), b2 = W.scorer_weights(cfg, std=0.03, bias_std=0.05)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16"), H.to_device(b1b, "bf16"), H.to_device(w2b, "bf16"), b2, B.STEP_BF16)
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (M, 8192), "bf16")
+    mask = W.boundary_mask(cfg, M, density=0.3)
+    rt = torch.from_numpy((np.arange(M) % T).astype(np.int32)).cuda()
+    got = pool.score_steps(H.to_device(hb, "bf16"), torch.from_numpy(mask).cuda(), rt, wts).cpu().numpy()
+    want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+    assert np.abs(got[mask == 1] - want[mask == 1]).max() <= 1e-3
+    pool.set_scorer_config(-1, 0)
+    with pytest.raises(B.StepError) as e:
+        pool.score_steps(H.to_device(hb, "bf16"), torch.from_numpy(mask).cuda(), rt, wts)
+    assert e.value.code == 1
