@@ -653,7 +653,7 @@ def run_scorer(args):
 
 # ---------------------------------------------------------------------------------------------
 def run_reference(args):
-    """The reference arm of this build is the CPU oracle, as it stands, on the host cores.
+    """The reference arm is the CPU oracle, as it stands, on the host cores.
     Under a multi-rank launcher rank 0 alone runs and prints; the other ranks leave at once."""
     from paper_2601_09093_b200 import ranks as R
     if R.rank_env()[0] != 0:

@@ -13,7 +13,7 @@ from gpu_common import Twin, exact_f32, attention_errors
 
 pytestmark = pytest.mark.gpu
 
-# tolerances stated by the benchmark spec for bf16-in / fp32-accumulate attention and for scores
+# tolerances for bf16-in / fp32-accumulate attention (max and mean absolute error) and for scores (absolute)
 ATT_MAX, ATT_MEAN, SCORE_TOL = 1e-2, 1e-3, 1e-3
 
 
