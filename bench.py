@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
     ap.add_argument("--scorer-density", type=float, default=1.0, help="fraction of those rows that end a step")
     ap.add_argument("--scorer-shape", default="c1", choices=["c1", "c4"])
+    ap.add_argument("--traces", type=int, default=0, help="c3 only: sampling budget N (traces sharing the pool); 0 = 64")
+    ap.add_argument("--threshold", type=float, default=0.0, help="c3 only: pool fraction at which the trigger fires; 0 = 0.95")
     ap.add_argument("--no-aux", action="store_true", help="skip the scorer / prune-cycle measurements after the timed steps")
     ap.add_argument("--num-blocks", type=int, default=0, help="override the pool size (blocks)")
     ap.add_argument("--grid", type=int, default=0, help="CTAs of the attention launch (0 = library default)")
@@ -112,11 +114,15 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------
-def workload_plan(name, num_blocks_override, steps_total, free_bytes=None):
+def workload_plan(name, num_blocks_override, steps_total, free_bytes=None, traces=0, threshold=0.0):
     """Shapes of the benchmark state: config, per-trace suffix lengths, pool size."""
     from paper_2601_09093_b200 import workloads as W
     if name == "c3":
         cfg = W.C3
+        if traces or threshold:
+            # the paper's sweeps: sampling budget N = 16 / 32 / 64 and the KV memory budget 0.5 - 0.9
+            cfg = W.scaled(cfg, n_traces=traces or cfg.n_traces, threshold=threshold or cfg.threshold,
+                           name="%s-N%d-thr%.2f" % (cfg.name, traces or cfg.n_traces, threshold or cfg.threshold))
         nb = num_blocks_override or cfg.num_blocks
         block_bytes = cfg.bytes_per_token * cfg.page_size
         if free_bytes is not None:
@@ -166,7 +172,8 @@ def run_ours(args):
     e2e_steps = 0 if args.no_e2e else K
     steps_total = Wm + K + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS + 3
     free_b, total_b = torch.cuda.mem_get_info(dev)
-    cfg, suffix, nb, max_pages, phys_layers = workload_plan(args.workload, args.num_blocks, steps_total, free_b)
+    cfg, suffix, nb, max_pages, phys_layers = workload_plan(args.workload, args.num_blocks, steps_total, free_b,
+                                                            args.traces, args.threshold)
     cfg_pool = W.scaled(cfg, num_layers=phys_layers)
     T, L = cfg.n_traces, cfg.num_layers
     pool = H.make_pool(cfg_pool, nb, max_pages, T, max_score_rows=T, device=dev)
@@ -515,7 +522,7 @@ def prune_cycles(pool, cfg, nb, T, dev, wts, append_log, phys_layers, hbm_peak, 
     for cyc in range(n_cycles):
         live_h = torch.nonzero(v["live"][:T]).flatten().cpu().tolist()
         n_live = len(live_h)
-        if n_live < 2:
+        if n_live < 4:                                                   # the block table is sized for four survivors
             break
         live = torch.tensor(live_h, dtype=torch.int32, device=dev)
         used = pool.stats()["used"]
@@ -665,7 +672,7 @@ def run_reference(args):
     K, Wm = args.steps, max(args.warmup, 1)
     if args.workload == "scorer":
         return run_reference_scorer(args, K, Wm)
-    cfg, suffix, nb, max_pages, _ = workload_plan(args.workload, args.num_blocks, Wm + K + 4)
+    cfg, suffix, nb, max_pages, _ = workload_plan(args.workload, args.num_blocks, Wm + K + 4, None, args.traces, args.threshold)
     T, L, P = cfg.n_traces, cfg.num_layers, cfg.page_size
     # bounded sample of one step: attention of ONE trace in ONE layer at the benchmark's length,
     # the scorer on the step's boundary rows, the pool bookkeeping and the trigger for all traces
