@@ -14,6 +14,8 @@
 //     16-byte chunk c stored at chunk c ^ (r % 8)); no compacted copy of the rows is ever made;
 //   * B = W1[n0 .. n0 + N, k .. k + 64): TMA tiled loads (one 64 x 64 box per 64 units, 128-byte
 //     swizzle) signalling the stage's mbarrier with their byte count;
+//   * the operand ring is 192 KiB; a stage holds exactly what the launch's item shape needs (24 KiB for 128 rows x
+//     64 units ... 64 KiB for 256 x 256), so small launches, which are latency-bound, get up to 8 stages in flight;
 //   * one thread issues tcgen05.mma (M 128, N 64 | 128 | 256, K 16) four times per row half and 64-wide k-chunk and
 //     commits the stage back to the producers;
 //   * eight warps read the finished accumulators with tcgen05.ld - a thread owns one row, so
@@ -34,13 +36,12 @@ namespace {
 constexpr int kHalfRows = 128;                    // UMMA M
 constexpr int kBK = 64;                           // bf16 elements per k-chunk (one 128-byte swizzle row)
 constexpr int kMaxN = 256;                        // UMMA N limit
-constexpr int kStages = 3;
+constexpr int kMaxStages = 8;
 constexpr int kHalfBytes = kHalfRows * kBK * 2;   // 16 KiB
-constexpr int kABytes = 2 * kHalfBytes;           // 32 KiB
+constexpr int kRingBytes = 192 * 1024;            // shared memory of the operand ring; a stage is as large as the
+                                                  // launch's item shape needs, so small shapes get more stages
 constexpr int kBoxRows = 64;                      // hidden units per TMA box
 constexpr int kBoxBytes = kBoxRows * kBK * 2;     // 8 KiB
-constexpr int kBBytes = kMaxN * kBK * 2;          // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;    // 64 KiB
 constexpr int kEpiWarps = 8, kGatherWarps = 8;    // read-out: warp w takes TMEM lanes 32 (w % 4) of accumulator w / 4
 constexpr int kWarpTma = kEpiWarps + kGatherWarps, kWarpMma = kWarpTma + 1;
 constexpr int kThreads = (kWarpMma + 1) * 32;     // 576
@@ -165,6 +166,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   const int slices = a.m / N;
   const int R = a.counters[C_SCORE_TILE];                       // rows per item: 256, or 128 for launches too small to
   const int tiles = (nb + R - 1) / R;                           // fill the SMs with 256-row items
+  // operand ring: a stage holds R x 64 of the hidden rows and N x 64 of W1 (24 - 64 KiB), 3 to 8 stages
+  const int a_bytes = R / kHalfRows * kHalfBytes;
+  const int stage_bytes = a_bytes + N * kBK * 2;
+  const int n_stages = min(kMaxStages, kRingBytes / stage_bytes);
   const int items = tiles * slices;
   const int KC = a.D / kBK;
 
@@ -172,18 +177,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles want 1024-byte alignment
   unsigned char* sm = smem_raw + (base - raw);
-  float* s_b1 = reinterpret_cast<float*>(sm + kStages * kStageBytes);
+  float* s_b1 = reinterpret_cast<float*>(sm + kRingBytes);
   float* s_w2 = s_b1 + kMaxUnits;
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_w2 + kMaxUnits);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 2);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kMaxStages + 2);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  const uint32_t bar_full = smem_u32(s_bar), bar_empty = bar_full + 8 * kStages;
-  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 8;
+  const uint32_t bar_full = smem_u32(s_bar), bar_empty = bar_full + 8 * kMaxStages;
+  const uint32_t bar_tfull = bar_empty + 8 * kMaxStages, bar_tempty = bar_tfull + 8;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(bar_full + 8 * s, kGatherWarps * 32 + 1);       // one arrival per gather thread + the TMA thread
       mbar_init(bar_empty + 8 * s, 1);                          // tcgen05.commit
     }
@@ -240,7 +245,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     const int tg = threadIdx.x - kEpiWarps * 32;                // 0 .. 255
     const int c = tg & 7, rb = tg >> 3;                         // 16-byte chunk of the row; rows rb + 32 i
     const uint32_t dst0 = base + (uint32_t)((rb >> 3) * 1024 + (rb & 7) * 128 + ((c ^ (rb & 7)) << 4));
-    int it = 0;
+    int s = 0;                                                  // ring position and its phase, kept incrementally
+    uint32_t ph = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
       const int tile = item / slices;
@@ -253,17 +259,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       }
       const int n_copy = R > kHalfRows && tile * R + kHalfRows < nb ? 8 : 4;   // the second half may be absent or empty
       int kr = first_chunk(item, KC);
-      for (int kc = 0; kc < KC; ++kc, ++it) {
-        const int s = it % kStages;
-        if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
-        const uint32_t dst = dst0 + (uint32_t)(s * kStageBytes);
+      for (int kc = 0; kc < KC; ++kc) {
+        if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ph ^ 1)) { ok = false; break; }
+        const uint32_t dst = dst0 + (uint32_t)(s * stage_bytes);
 #pragma unroll
         for (int i = 0; i < 8; ++i)
           if (i < n_copy) cp_async16(dst + i * 4096, src[i] + kr * kBK);
         if (++kr == KC) kr = 0;
         // the stage's barrier hears from this thread when these copies have landed; the thread moves on at once,
-        // so the copies of up to kStages chunks are in flight and nothing here waits for data
+        // so the copies of all stages can be in flight and nothing here waits for data
         cp_async_arrive_when_done(bar_full + 8 * s);
+        if (++s == n_stages) { s = 0; ph ^= 1; }
       }
     }
     cp_async_wait_all();                                        // nothing of this thread is in flight when it leaves
@@ -274,29 +280,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   } else if (warp == kWarpTma) {
     // ------------------------------------------------ TMA loads of the W1 slice into B
     if (lane == 0) {
-      int it = 0;
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
       const int boxes = N / kBoxRows;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
         const int n0 = (item % slices) * N;
         int kr = first_chunk(item, KC);
-        for (int kc = 0; kc < KC; ++kc, ++it) {
-          const int s = it % kStages;
-          if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { ok = false; break; }
+        for (int kc = 0; kc < KC; ++kc) {
+          if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ph ^ 1)) { ok = false; break; }
           const uint32_t bar = bar_full + 8 * s;
           mbar_expect_tx(bar, (uint32_t)(boxes * kBoxBytes));
-          const uint32_t dst = base + (uint32_t)(s * kStageBytes + kABytes);
+          const uint32_t dst = base + (uint32_t)(s * stage_bytes + a_bytes);
           for (int j = 0; j < boxes; ++j) tma_load_2d(dst + j * kBoxBytes, &map_w1, kr * kBK, n0 + j * kBoxRows, bar);
           if (++kr == KC) kr = 0;
+          if (++s == n_stages) { s = 0; ph ^= 1; }
         }
       }
       if (!ok) {
         flag_error(a.counters, STEP_ERR_TIMEOUT);
         *s_abort = 1;
         // loads already issued still target this CTA's shared memory: give them a moment to land
-        for (int s = 0; s < kStages; ++s) {
-          mbar_wait_bounded(bar_full + 8 * s, 0, kDrainNs);
-          mbar_wait_bounded(bar_full + 8 * s, 1, kDrainNs);
+        for (int q = 0; q < n_stages; ++q) {
+          mbar_wait_bounded(bar_full + 8 * q, 0, kDrainNs);
+          mbar_wait_bounded(bar_full + 8 * q, 1, kDrainNs);
         }
       }
     }
@@ -305,7 +312,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     // ------------------------------------------------ MMA issue
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(N);
-      int it = 0, li = 0;
+      int s = 0, li = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++li) {
         const int tile = item / slices;
@@ -313,20 +321,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
         // the read-out of the previous item must have drained the accumulators
         if (*s_abort || !mbar_wait_bounded(bar_tempty, (li & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
-        for (int kc = 0; kc < KC; ++kc, ++it) {
-          const int s = it % kStages;
-          if (*s_abort || !mbar_wait_bounded(bar_full + 8 * s, (it / kStages) & 1)) { ok = false; break; }
+        for (int kc = 0; kc < KC; ++kc) {
+          if (*s_abort || !mbar_wait_bounded(bar_full + 8 * s, ph)) { ok = false; break; }
           fence_async_smem();                                   // the gathered rows were written through the generic proxy
           tc_fence_after();
-          const uint64_t bdesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + kABytes));
+          const uint64_t bdesc = umma_desc_sw128(base + (uint32_t)(s * stage_bytes + a_bytes));
           for (int h = 0; h < halves; ++h) {                    // both row halves multiply the same W1 tile
-            const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * kStageBytes + h * kHalfBytes));
+            const uint64_t adesc = umma_desc_sw128(base + (uint32_t)(s * stage_bytes + h * kHalfBytes));
             const uint32_t d_tmem = tmem_base + (uint32_t)(h * kMaxN);
 #pragma unroll
             for (int kk = 0; kk < kBK / 16; ++kk)                // 16 bf16 = 32 bytes further along the swizzled row
               tc_mma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kc | kk) != 0);
           }
           tc_commit(bar_empty + 8 * s);                         // the stage is free once these products have read it
+          if (++s == n_stages) { s = 0; ph ^= 1; }
         }
         if (ok) tc_commit(bar_tfull);                           // the accumulators are complete
       }
@@ -346,8 +354,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   }
 }
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 2 * kMaxUnits * sizeof(float) +
-                              (2 * kStages + 2) * sizeof(uint64_t) + 16;
+constexpr size_t kSmemBytes = 1024 + (size_t)kRingBytes + 2 * kMaxUnits * sizeof(float) +
+                              (2 * kMaxStages + 2) * sizeof(uint64_t) + 16;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
