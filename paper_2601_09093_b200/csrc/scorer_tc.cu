@@ -28,6 +28,7 @@
 #include "step_internal.cuh"
 
 #include <cuda.h>
+#include <string.h>
 
 using namespace stepk;
 
@@ -253,18 +254,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       const __nv_bfloat16* src[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        int gr = tile * R + rb + 32 * i;
-        if (gr >= nb) gr = nb - 1;                              // rows past the list re-read its last row; never stored
-        src[i] = a.hidden + (size_t)a.idx[gr] * a.D + c * 8;
+        const int gr = tile * R + rb + 32 * i;
+        // rows past the end of the list are not fetched: each output row depends on its own operand row only, so
+        // whatever the shared memory holds there ends up in accumulator rows that nobody reads out
+        src[i] = gr < nb && 32 * i < R ? a.hidden + (size_t)a.idx[gr] * a.D + c * 8 : nullptr;
       }
-      const int n_copy = R > kHalfRows && tile * R + kHalfRows < nb ? 8 : 4;   // the second half may be absent or empty
       int kr = first_chunk(item, KC);
       for (int kc = 0; kc < KC; ++kc) {
         if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ph ^ 1)) { ok = false; break; }
         const uint32_t dst = dst0 + (uint32_t)(s * stage_bytes);
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (i < n_copy) cp_async16(dst + i * 4096, src[i] + kr * kBK);
+          if (src[i]) cp_async16(dst + i * 4096, src[i] + kr * kBK);
         if (++kr == KC) kr = 0;
         // the stage's barrier hears from this thread when these copies have landed; the thread moves on at once,
         // so the copies of all stages can be in flight and nothing here waits for data
@@ -388,20 +389,30 @@ bool score_tc_supported(const scorer_weights* w, const void* hidden) {
   return encode_tiled_fn() != nullptr;
 }
 
-int score_tc_launch(const step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s) {
-  EncodeTiledFn enc = encode_tiled_fn();
-  if (!enc) return STEP_ERR_CUDA;
+int score_tc_launch(step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s) {
+  static_assert(sizeof(CUtensorMap) <= sizeof(pool->tmap_bytes), "tensor map cache too small");
+  if (pool->tmap_w1 != w->W1 || pool->tmap_D != w->D || pool->tmap_m != w->m) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return STEP_ERR_CUDA;
+    CUtensorMap fresh;
+    const cuuint64_t dims[2] = {(cuuint64_t)w->D, (cuuint64_t)w->m};       // innermost first
+    const cuuint64_t strides[1] = {(cuuint64_t)w->D * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kBoxRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&fresh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w->W1), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return STEP_ERR_CUDA;
+    memcpy(pool->tmap_bytes, &fresh, sizeof(fresh));
+    pool->tmap_w1 = w->W1; pool->tmap_D = w->D; pool->tmap_m = w->m;
+  }
   CUtensorMap map;
-  const cuuint64_t dims[2] = {(cuuint64_t)w->D, (cuuint64_t)w->m};       // innermost first
-  const cuuint64_t strides[1] = {(cuuint64_t)w->D * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kBoxRows};
-  const cuuint32_t estr[2] = {1, 1};
-  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w->W1), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return STEP_ERR_CUDA;
-  if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
-    return STEP_ERR_CUDA;
+  memcpy(&map, pool->tmap_bytes, sizeof(map));
+  if (!pool->tc_smem_set) {
+    if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+      return STEP_ERR_CUDA;
+    pool->tc_smem_set = true;
+  }
   TcArgs a;
   a.hidden = (const __nv_bfloat16*)hidden;
   a.b1 = (const __nv_bfloat16*)w->b1; a.w2 = (const __nv_bfloat16*)w->w2;

@@ -69,6 +69,10 @@ struct step_pool {
   int fast_path;      // 1 allowed, -1 forced off
   int scorer_mode;    // 0: tensor-core MLP for launches with >= scorer_tc_min_rows boundary rows; 1: always; -1: never
   int scorer_tc_min_rows;
+  // the tensor map of the last W1 the tensor-core scorer was given (encoding it costs a few host microseconds)
+  alignas(64) unsigned char tmap_bytes[128];
+  const void* tmap_w1; int tmap_D, tmap_m;
+  bool tc_smem_set;   // the scorer kernel's dynamic shared memory limit has been raised on this pool's device
   int device;
   stepk::MetaLayout lay;
   stepk::DevViews v;
@@ -138,6 +142,6 @@ int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const 
 bool score_tc_supported(const scorer_weights* w, const void* hidden);
 // Launches the persistent kernel for a chunk of Mc candidate rows (at most one CTA per SM); it reads
 // C_SCORE_NB / C_SCORE_TC on the device and returns at once when C_SCORE_TC is 0.
-int score_tc_launch(const step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s);
+int score_tc_launch(step_pool* pool, const void* hidden, int Mc, const scorer_weights* w, cudaStream_t s);
 
 }  // namespace stepk
