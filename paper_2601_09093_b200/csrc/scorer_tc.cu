@@ -171,7 +171,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   const int a_bytes = R / kHalfRows * kHalfBytes;
   const int stage_bytes = a_bytes + N * kBK * 2;
   const int n_stages = min(kMaxStages, kRingBytes / stage_bytes);
-  const int items = tiles * slices;
+  // Items are handed out round-robin, so a launch takes as long as the CTA with the most items.  With 256-row
+  // items the last round can be nearly empty; the rows that would make it up are cut into 128-row items instead,
+  // which spreads that last bit of work over twice as many CTAs.  (The ring keeps the 256-row stage layout.)
+  int n_big = tiles * slices, n_big_tiles = tiles, n_small = 0;
+  if (R > kHalfRows && n_big > (int)gridDim.x && n_big % (int)gridDim.x != 0) {
+    n_big_tiles = n_big / (int)gridDim.x * (int)gridDim.x / slices;
+    n_big = n_big_tiles * slices;
+    n_small = (nb - n_big_tiles * R + kHalfRows - 1) / kHalfRows * slices;
+  }
+  const int items = n_big + n_small;
+  // item -> first listed row, rows (256 or 128), slice of hidden units
+  auto item_rows = [&](int item, int& row0, int& slice) -> int {
+    if (item < n_big) { const int t = item / slices; slice = item - t * slices; row0 = t * R; return R; }
+    const int j = item - n_big, t = j / slices;
+    slice = j - t * slices; row0 = n_big_tiles * R + t * kHalfRows;
+    return kHalfRows;
+  };
   const int KC = a.D / kBK;
 
   extern __shared__ unsigned char smem_raw[];
@@ -216,7 +232,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     const int quarter = warp & 3, half = warp >> 2;
     int li = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, ++li) {
-      const int tile = item / slices, slice = item - tile * slices, n0 = slice * N;
+      int row0, slice;
+      const int rows = item_rows(item, row0, slice);
+      const int n0 = slice * N;
       if (*s_abort) break;
       if (!mbar_wait_bounded(bar_tfull, li & 1)) {
         if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
@@ -224,8 +242,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
         break;
       }
       tc_fence_after();
-      const int row = tile * R + half * kHalfRows + quarter * 32 + lane;
-      const bool used = half * kHalfRows < R && tile * R + half * kHalfRows < nb;   // did this half get any products?
+      const int row = row0 + half * kHalfRows + quarter * 32 + lane;
+      const bool used = half * kHalfRows < rows && row0 + half * kHalfRows < nb;    // did this half get any products?
       float z = 0.f;
       if (used) {
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * kMaxN);
@@ -250,14 +268,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     uint32_t ph = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
-      const int tile = item / slices;
+      int row0, slice;
+      const int rows = item_rows(item, row0, slice);
       const __nv_bfloat16* src[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const int gr = tile * R + rb + 32 * i;
+        const int gr = row0 + rb + 32 * i;
         // rows past the end of the list are not fetched: each output row depends on its own operand row only, so
         // whatever the shared memory holds there ends up in accumulator rows that nobody reads out
-        src[i] = gr < nb && 32 * i < R ? a.hidden + (size_t)a.idx[gr] * a.D + c * 8 : nullptr;
+        src[i] = gr < nb && 32 * i < rows ? a.hidden + (size_t)a.idx[gr] * a.D + c * 8 : nullptr;
       }
       int kr = first_chunk(item, KC);
       for (int kc = 0; kc < KC; ++kc) {
@@ -286,7 +305,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       bool ok = true;
       const int boxes = N / kBoxRows;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
-        const int n0 = (item % slices) * N;
+        int row0, slice;
+        item_rows(item, row0, slice);
+        const int n0 = slice * N;
         int kr = first_chunk(item, KC);
         for (int kc = 0; kc < KC; ++kc) {
           if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ph ^ 1)) { ok = false; break; }
@@ -317,8 +338,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       uint32_t ph = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++li) {
-        const int tile = item / slices;
-        const int halves = R > kHalfRows && tile * R + kHalfRows < nb ? 2 : 1;
+        int row0, slice;
+        const int rows = item_rows(item, row0, slice);
+        const int halves = rows > kHalfRows && row0 + kHalfRows < nb ? 2 : 1;
         // the read-out of the previous item must have drained the accumulators
         if (*s_abort || !mbar_wait_bounded(bar_tempty, (li & 1) ^ 1)) { ok = false; break; }
         tc_fence_after();
