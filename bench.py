@@ -216,7 +216,7 @@ def run_ours(args):
 
     ids_host = list(ids)
 
-    def hot_path(s, time_attn=False):
+    def hot_path(s, time_attn=False, out=out, step_scores=step_scores):
         pool.append_kv(ids_dev, 1, s["k"], s["v"])
         append_log.append((ids_host, 1))
         for l in range(L):
@@ -229,15 +229,60 @@ def run_ours(args):
         pool.score_steps(s["h"], s["m"], None, wts, step_scores)
         pool.prune_if_saturated(None, cfg.threshold, cfg.keep_frac)
 
-    def e2e_step(s, dst):
-        for k in ("q", "k", "v", "h", "m"):
-            dst[k].copy_(s["host"][k], non_blocking=True)
-        hot_path(dst)
-        host_out.copy_(out, non_blocking=True)
-        host_scores.copy_(step_scores, non_blocking=True)
-        host_tscores.copy_(v["trace_scores"], non_blocking=True)
-        host_npruned.copy_(pool.n_pruned, non_blocking=True)
-        stream.synchronize()
+    def make_e2e():
+        """Returns run(n_steps): n_steps steps whose inputs start in pinned host memory and whose results end there,
+        software-pipelined the way a serving loop would: while step i computes, the copy engines bring in the inputs of step i + 1 and take
+        out the results of step i - 1 (two sets of device and host buffers); the host reads a step's results one step
+        late.  Every step's copies happen inside the region that is timed; the buffers are set up here, outside it."""
+        h2d_s, d2h_s = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        keys = ("q", "k", "v", "h", "m")
+        dst = [{k: torch.empty_like(sets[0][k]) for k in keys} for _ in range(2)]
+        outs = [out, torch.empty_like(out)]
+        sc = [step_scores, torch.empty_like(step_scores)]
+        ts = [torch.empty(pool.max_traces, dtype=torch.float32, device=dev) for _ in range(2)]
+        npr = [torch.empty(1, dtype=torch.int32, device=dev) for _ in range(2)]
+        host = [dict(out=host_out, sc=host_scores, ts=host_tscores, n=host_npruned),
+                dict(out=torch.empty_like(host_out).pin_memory(), sc=torch.empty_like(host_scores).pin_memory(),
+                     ts=torch.empty_like(host_tscores).pin_memory(), n=torch.empty_like(host_npruned).pin_memory())]
+        in_done = [torch.cuda.Event() for _ in range(2)]
+        comp_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
+
+        def run(n_steps):
+            fetch(0)
+            for i in range(n_steps):
+                p = i % 2
+                if i + 1 < n_steps:
+                    fetch(i + 1)
+                stream.wait_event(in_done[p])
+                if i >= 2:
+                    stream.wait_event(out_done[p])      # the results of step i - 2 have left these buffers
+                hot_path(dst[p], out=outs[p], step_scores=sc[p])
+                ts[p].copy_(v["trace_scores"], non_blocking=True)
+                npr[p].copy_(pool.n_pruned, non_blocking=True)
+                comp_done[p].record(stream)
+                with torch.cuda.stream(d2h_s):
+                    d2h_s.wait_event(comp_done[p])
+                    host[p]["out"].copy_(outs[p], non_blocking=True)
+                    host[p]["sc"].copy_(sc[p], non_blocking=True)
+                    host[p]["ts"].copy_(ts[p], non_blocking=True)
+                    host[p]["n"].copy_(npr[p], non_blocking=True)
+                    out_done[p].record(d2h_s)
+                if i >= 1:
+                    out_done[1 - p].synchronize()       # the host has step i - 1's results
+            out_done[(n_steps - 1) % 2].synchronize()
+            torch.cuda.synchronize()
+
+        def fetch(i):                                   # inputs of step i -> device set i % 2
+            p = i % 2
+            with torch.cuda.stream(h2d_s):
+                if i >= 2:
+                    h2d_s.wait_event(comp_done[p])      # step i - 2 has finished reading this set
+                for k in keys:
+                    dst[p][k].copy_(sets[i % NSETS]["host"][k], non_blocking=True)
+                in_done[p].record(h2d_s)
+
+        return run
 
     def barrier():
         torch.cuda.synchronize()
@@ -268,13 +313,11 @@ def run_ours(args):
     # ---- end to end: host buffers in, host results out, every step
     e2e = None
     if e2e_steps:
-        dst = {k: torch.empty_like(sets[0][k]) for k in ("q", "k", "v", "h", "m")}
-        for i in range(Wm):
-            e2e_step(sets[i % NSETS], dst)
+        e2e_run = make_e2e()
+        e2e_run(Wm)
         barrier()
         t0 = time.perf_counter()
-        for i in range(e2e_steps):
-            e2e_step(sets[i % NSETS], dst)
+        e2e_run(e2e_steps)
         barrier()
         e2e_s = time.perf_counter() - t0
         h2d = sum(sets[0]["host"][k].numel() * sets[0]["host"][k].element_size() for k in ("q", "k", "v", "h", "m"))
