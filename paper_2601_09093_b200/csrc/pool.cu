@@ -209,30 +209,36 @@ __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict
   }
 }
 
-// Phase 2: one thread moves one 16-byte chunk of a new K or V row into its page.
-__global__ void append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ knew,
-                                    const uint4* __restrict__ vnew, const int32_t* __restrict__ ids,
-                                    int n, int n_tokens, int cpr, int cpe, int src_by_id) {
-  const size_t per_kv = (size_t)n * n_tokens * g.L * g.Hkv * cpr;
-  const size_t total = per_kv * 2;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+// Phase 2: the new rows go into their pages.  A CTA owns one (listed trace, new token) pair and a range of
+// layers: where the token lands (page, slot, block) is worked out once per CTA, and per layer the threads move the
+// 16-byte chunks of the K and V rows of all KV heads with nothing but adds in the loop.
+// grid (n * n_tokens, layer splits).
+__global__ void __launch_bounds__(256)
+append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ knew,
+                    const uint4* __restrict__ vnew, const int32_t* __restrict__ ids,
+                    int n_tokens, int cpr, int layers_per_cta, int src_by_id) {
+  const int idx = blockIdx.x / n_tokens, j = blockIdx.x - idx * n_tokens;
+  const int base = v.append_base[idx];
+  if (base < 0) return;                                          // this trace's request was not met
+  const int t = ids[idx];
+  const int pos = base + j, page = pos / g.P, slot = pos % g.P;
+  const int b = v.block_table[(size_t)t * g.max_pages + page];
+  const int l0 = blockIdx.y * layers_per_cta, l1 = min(g.L, l0 + layers_per_cta);
+  const int per_kv = g.Hkv * cpr;                                // chunks of the K (or V) rows of one layer
+  // the new rows are laid out [row, token, layer, head, chunk]; row = position in the list, or the trace id
+  const size_t row = src_by_id ? (size_t)t : (size_t)idx;
+  const size_t src_token = (row * n_tokens + j) * (size_t)g.L * per_kv;
+  const size_t page_chunks = (size_t)g.P * cpr;                  // 16-byte chunks of one K (or V) page
+  for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
     const int which = i >= per_kv;
-    const size_t src = which ? i - per_kv : i;
-    size_t r = src;
-    const int c = r % cpr; r /= cpr;
-    const int head = r % g.Hkv; r /= g.Hkv;
-    const int layer = r % g.L; r /= g.L;
-    const int j = r % n_tokens; const int idx = r / n_tokens;
-    const int base = v.append_base[idx];
-    if (base < 0) continue;
-    const int t = ids[idx];
-    const int pos = base + j, page = pos / g.P, slot = pos % g.P;
-    const int b = v.block_table[(size_t)t * g.max_pages + page];
+    const int r = which ? i - per_kv : i;
+    const int head = r / cpr, c = r - head * cpr;
     const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
-    const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
-    // the new rows are laid out [row, token, layer, head, chunk]; row = position in the list, or the trace id
-    const size_t from = src_by_id ? ((((size_t)t * n_tokens + j) * g.L + layer) * g.Hkv + head) * cpr + c : src;
-    kv[e / cpe + cdst] = (which ? vnew : knew)[from];
+    const uint4* src = (which ? vnew : knew) + src_token + r;
+    // chunk index of (layer, b, head, which, slot, cdst): pages are [layer][block][head][K|V]
+    const size_t dst0 = (((size_t)b * g.Hkv + head) * 2 + which) * page_chunks + (size_t)slot * cpr + cdst;
+    const size_t layer_stride = (size_t)g.num_blocks * g.Hkv * 2 * page_chunks;
+    for (int l = l0; l < l1; ++l) kv[(size_t)l * layer_stride + dst0] = src[(size_t)l * per_kv];
   }
 }
 
@@ -389,9 +395,17 @@ int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int 
     if (n_dev && off > 0) return STEP_ERR_INVALID_ARG;              // a device-side count covers one launch only
     append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens, n_dev);
     const size_t src_off = src_by_id ? 0 : row_chunks * off;
-    append_write_kernel<<<grid_for(row_chunks * m * 2, 256, pool->num_sms), 256, 0, s>>>(
+    // enough CTAs to occupy the device: (trace, token) pairs x splits of the layer range
+    const long long pairs = (long long)m * n_tokens;
+    if (pairs > 0x7fffffffll) return STEP_ERR_INVALID_ARG;
+    int splits = (int)((2ll * pool->num_sms + pairs - 1) / pairs);
+    if (splits > g.L) splits = g.L;
+    if (splits < 1) splits = 1;
+    const int layers_per_cta = (g.L + splits - 1) / splits;
+    splits = (g.L + layers_per_cta - 1) / layers_per_cta;
+    append_write_kernel<<<dim3((unsigned)pairs, (unsigned)splits), 256, 0, s>>>(
         pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off,
-        (const uint4*)v_new + src_off, trace_ids + off, m, n_tokens, cpr, cpe, src_by_id);
+        (const uint4*)v_new + src_off, trace_ids + off, n_tokens, cpr, layers_per_cta, src_by_id);
   }
   return launch_ok();
 }
