@@ -122,28 +122,31 @@ __global__ void fork_alloc_kernel(DevViews v, Geo g, int first_trace, int n_trac
   if (threadIdx.x == 0) v.counters[C_FREE_COUNT] = fc - needed;
 }
 
-// One thread moves one 16-byte chunk of the prompt's K or V.
-__global__ void fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ kpre,
-                                  const uint4* __restrict__ vpre, int first_trace, int n_traces,
-                                  int prefix_len, int cpr /*chunks per row*/, int cpe) {
+// The prompt's K and V rows go into their pages.  A CTA owns one prompt position and a range of layers; the
+// position's block (one shared block, or one private block per trace for a partial last page) is looked up once.
+// k_prefix, v_prefix: [layer, head, position, chunk].  grid (prefix_len, layer splits).
+__global__ void __launch_bounds__(256)
+fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ kpre,
+                  const uint4* __restrict__ vpre, int first_trace, int n_traces, int prefix_len, int cpr,
+                  int layers_per_cta) {
   if (!v.counters[C_FORK_OK]) return;
-  const int full = prefix_len / g.P;
-  const size_t per_kv = (size_t)g.L * g.Hkv * prefix_len * cpr;
-  const size_t total = per_kv * 2;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+  const int pos = blockIdx.x, page = pos / g.P, slot = pos % g.P;
+  const int copies = page < prefix_len / g.P ? 1 : n_traces;     // the partial page is private per trace
+  const int l0 = blockIdx.y * layers_per_cta, l1 = min(g.L, l0 + layers_per_cta);
+  const int per_kv = g.Hkv * cpr;
+  const size_t page_chunks = (size_t)g.P * cpr;
+  const size_t layer_stride = (size_t)g.num_blocks * g.Hkv * 2 * page_chunks;
+  for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
     const int which = i >= per_kv;
-    size_t r = which ? i - per_kv : i;
-    const int c = r % cpr; r /= cpr;
-    const int pos = r % prefix_len; r /= prefix_len;
-    const int head = r % g.Hkv; const int layer = r / g.Hkv;
-    const uint4 val = (which ? vpre : kpre)[i - (which ? per_kv : 0)];
-    const int page = pos / g.P, slot = pos % g.P;
+    const int r = which ? i - per_kv : i;
+    const int head = r / cpr, c = r - head * cpr;
     const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
-    const int copies = page < full ? 1 : n_traces;     // the partial page is private per trace
+    const uint4* src = (which ? vpre : kpre) + ((size_t)head * prefix_len + pos) * cpr + c;
+    const size_t src_layer = (size_t)g.Hkv * prefix_len * cpr;
     for (int j = 0; j < copies; ++j) {
       const int b = v.block_table[(size_t)(first_trace + j) * g.max_pages + page];
-      const size_t e = kv_page_base(g, layer, b, head, which) + (size_t)slot * g.d;
-      kv[e / cpe + cdst] = val;
+      const size_t dst0 = (((size_t)b * g.Hkv + head) * 2 + which) * page_chunks + (size_t)slot * cpr + cdst;
+      for (int l = l0; l < l1; ++l) kv[(size_t)l * layer_stride + dst0] = src[(size_t)l * src_layer];
     }
   }
 }
@@ -363,10 +366,14 @@ int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const voi
   fork_alloc_kernel<<<1, 256, 0, s>>>(pool->v, g, first, n_traces, prefix_len);
   if (prefix_len > 0) {
     const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
-    size_t chunks = (size_t)g.L * g.Hkv * prefix_len * cpr * 2;
-    fork_write_kernel<<<grid_for(chunks, 256, pool->num_sms), 256, 0, s>>>(
+    int splits = (2 * pool->num_sms + prefix_len - 1) / prefix_len;
+    if (splits > g.L) splits = g.L;
+    if (splits < 1) splits = 1;
+    const int layers_per_cta = (g.L + splits - 1) / splits;
+    splits = (g.L + layers_per_cta - 1) / layers_per_cta;
+    fork_write_kernel<<<dim3((unsigned)prefix_len, (unsigned)splits), 256, 0, s>>>(
         pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_prefix, (const uint4*)v_prefix, first,
-        n_traces, prefix_len, cpr, cpe);
+        n_traces, prefix_len, cpr, layers_per_cta);
   }
   pool->next_trace += n_traces;
   if (trace_ids_out) for (int j = 0; j < n_traces; ++j) trace_ids_out[j] = first + j;
