@@ -25,3 +25,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """libstep.so is built in-tree (nvcc, a no-op when it is up to date) before any test loads it."""
+    from paper_2601_09093_b200 import build
+    build.build()
