@@ -327,9 +327,12 @@ def run_ours(args):
     (ms_total, e2e_max), all_ok = R.max_over_ranks([ms_total, e2e[0] if e2e else 0.0], err_mask == 0 and n_live == T, dev)
     if e2e:
         e2e = (e2e_max, e2e[1], e2e[2])
+    if world > 1:
+        # every rank leaves the group at the same point; the CPU baseline and the measurements that follow the timed
+        # steps belong to single-GPU runs (they would hold the other GPUs idle)
+        dist.destroy_process_group()
+        args.no_cpu_baseline = args.no_aux = True
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
         return
 
     # ---- roofline of the dominant kernel (decode_attention of one layer)
@@ -378,8 +381,6 @@ def run_ours(args):
             if not args.no_cpu_baseline:
                 res["prune_cycles"]["oracle_replay"] = replay_cycles_on_oracle(cfg, nb, T, max_pages, append_log, cyc["snapshots"])
     print(json.dumps(res))
-    if world > 1:
-        dist.destroy_process_group()
 
 
 def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0):
