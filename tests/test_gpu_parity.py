@@ -134,7 +134,7 @@ def test_c0_attention_fp32():
     _check_attention(tw, cfg, cfg.n_traces, max_tol=1e-4, mean_tol=1e-5)
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (64, 8), (8, 8), (16, 1), (24, 2)])
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (64, 8), (8, 8), (16, 1), (24, 2), (40, 10)])
 def test_bf16_attention_ragged_small(Hq, Hkv):
     # several pages per warp partition, partial last pages, a one-token and an empty trace
     cfg = W.scaled(W.C1, n_traces=9, num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=48)
