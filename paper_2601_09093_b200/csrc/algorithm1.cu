@@ -53,6 +53,7 @@ finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, const i
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ int s_warp[33];
+  if (n_dev && *n_dev <= 0) return;      // nobody completes (every CTA reads the same count: the whole cluster leaves)
   if (cluster.block_rank() == 0) {
     const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
     int k = 0;
