@@ -277,6 +277,31 @@ typedef struct {
  * live trace do nothing) or max_iterations, then the weighted vote.  res is a HOST struct; synchronises. */
 int algorithm1_run(step_pool* pool, const step_run_args* args, step_run_result* res, void* stream);
 
+/* ---- training the step scorer (Sec. 3.1 "Training Objective"; appendix "Training Parameters") ----
+ * One optimisation step on a batch of B (hidden state, label) pairs:
+ *   L = -(1/B) sum_b ( pos_weight * y_b * log yhat_b + (1 - y_b) * log(1 - yhat_b) ),  yhat = f(h),
+ * pos_weight = alpha = K- / K+ (negative over positive samples of the training set); then Adam with the weight decay
+ * added to the gradient (g += weight_decay * p) and bias-corrected moments.  The paper's values: B = 128,
+ * lr = 1e-4, weight_decay = 1e-5; beta1 = 0.9, beta2 = 0.999, eps = 1e-8 are the optimiser's usual defaults (the
+ * paper does not list them).  `step` is the 1-based number of this update (for the bias correction). */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay, pos_weight;
+  int step;
+} scorer_train_hyper;
+
+/* Bytes of device workspace scorer_train_step needs (pre-activations and gradients); host-only, 0 on bad arguments. */
+size_t scorer_train_workspace_bytes(int B, int D, int m);
+
+/* hidden: [B, D] in hidden_dtype (STEP_BF16 | STEP_FP32); labels: [B] fp32 in {0, 1}; W1 [m, D], b1 [m], w2 [m],
+ * b2 [1]: fp32 parameters, updated in place; adam_m, adam_v: [m*D + 2m + 1] fp32 moments in the order W1, b1, w2, b2
+ * (zero before the first step), updated in place; workspace: 256-byte aligned, at least
+ * scorer_train_workspace_bytes(B, D, m); loss_out: [1] fp32, the loss BEFORE the update.  All device pointers except
+ * `h`.  Asynchronous on the stream; deterministic. */
+int scorer_train_step(const void* hidden, int hidden_dtype, const float* labels, int B, float* W1, float* b1,
+                      float* w2, float* b2, int D, int m, float* adam_m, float* adam_v,
+                      const scorer_train_hyper* h, void* workspace, size_t workspace_bytes, float* loss_out,
+                      void* stream);
+
 /* ---- accessors for tests and benchmarks ---- */
 /* Vote state: final_score [max_traces] f32, answer [max_traces] i32, finished [max_traces] u8 (device). */
 int kv_pool_vote_views(step_pool* pool, float** final_score, int32_t** answer, uint8_t** finished);

@@ -65,6 +65,11 @@ class step_run_result(C.Structure):
                 ("n_finished", C.c_int), ("n_evicted", C.c_int), ("live_left", C.c_int)]
 
 
+class scorer_train_hyper(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("pos_weight", C.c_float), ("step", C.c_int)]
+
+
 _lib = None
 
 
@@ -99,6 +104,9 @@ def lib():
     L.kv_pool_last_error.argtypes = [vp, C.POINTER(C.c_uint), vp]
     L.kv_pool_read_kv.argtypes = [vp, i, i, vp, i, vp, vp, vp]
     L.kv_pool_set_attention_config.argtypes = [vp, i, i]
+    L.scorer_train_workspace_bytes.argtypes = [i, i, i]
+    L.scorer_train_workspace_bytes.restype = C.c_size_t
+    L.scorer_train_step.argtypes = [vp, i, vp, i, vp, vp, vp, vp, i, i, vp, vp, C.POINTER(scorer_train_hyper), vp, C.c_size_t, vp, vp]
     L.kv_pool_finish_traces.argtypes = [vp, vp, vp, i, vp]
     L.weighted_vote.argtypes = [vp, vp, vp, vp, vp]
     L.kv_pool_vote_views.argtypes = [vp] + [C.POINTER(vp)] * 3
@@ -347,6 +355,35 @@ class KVPool:
         n, u = C.c_int(), C.c_int()
         _check("kv_pool_score_launch_info", lib().kv_pool_score_launch_info(self.handle, C.byref(n), C.byref(u), _stream(stream)))
         return dict(n_rows=n.value, tc_units=u.value)
+
+
+class ScorerTrainer:
+    """fp32 scorer parameters, Adam moments and workspace on the device; step() forwards to scorer_train_step."""
+
+    def __init__(self, W1, b1, w2, b2, batch, lr=1e-4, weight_decay=1e-5, pos_weight=1.0, beta1=0.9, beta2=0.999, eps=1e-8):
+        self.W1, self.b1, self.w2 = (x.to(torch.float32, copy=True).contiguous() for x in (W1, b1, w2))   # owned copies
+        self.b2 = torch.tensor([float(b2)], dtype=torch.float32, device=self.W1.device)
+        self.m, self.D = self.W1.shape
+        n = self.m * self.D + 2 * self.m + 1
+        self.adam_m = torch.zeros(n, dtype=torch.float32, device=self.W1.device)
+        self.adam_v = torch.zeros_like(self.adam_m)
+        self.batch = batch
+        self.ws_bytes = lib().scorer_train_workspace_bytes(batch, self.D, self.m)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.W1.device)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=self.W1.device)
+        self.h = scorer_train_hyper(lr=lr, beta1=beta1, beta2=beta2, eps=eps, weight_decay=weight_decay,
+                                    pos_weight=pos_weight, step=0)
+
+    def step(self, hidden, labels, stream=None):
+        """One update; returns the device tensor holding the loss before the update (no sync)."""
+        assert hidden.shape == (self.batch, self.D) and labels.dtype == torch.float32
+        self.h.step += 1
+        dt = STEP_BF16 if hidden.dtype == torch.bfloat16 else STEP_FP32
+        _check("scorer_train_step", lib().scorer_train_step(
+            _ptr(hidden), dt, _ptr(labels), self.batch, _ptr(self.W1), _ptr(self.b1), _ptr(self.w2), _ptr(self.b2),
+            self.D, self.m, _ptr(self.adam_m), _ptr(self.adam_v), C.byref(self.h), _ptr(self.ws), self.ws_bytes,
+            _ptr(self.loss), _stream(stream)))
+        return self.loss
 
 
 def step_end_table_from_vocab(token_texts):
