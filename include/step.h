@@ -120,6 +120,20 @@ int decode_attention(step_pool* pool, int layer, const void* q,
                      const int32_t* block_table, const int32_t* seq_lens, int n,
                      void* out, void* stream);
 
+/* decode_attention for traces that share their first pages (the prompt pages kv_pool_fork_prefix allocates once for
+ * all traces of a problem: Algorithm 1, InitTraces):
+ *   out[i] = attention of q[i] over the prefix_pages * page_size positions stored in blocks prefix_blocks[0 ..
+ *            prefix_pages) followed by positions [prefix_pages * page_size, seq_lens[i]) of row i of block_table,
+ * which is decode_attention's result whenever block_table[i][p] == prefix_blocks[p] for every listed row and
+ * p < prefix_pages (prefix_blocks may point at any such row).  The shared pages are read once per 16 / G traces
+ * instead of once per trace.  prefix_blocks: [prefix_pages] int32, device.  prefix_pages = 0 is decode_attention.
+ * A row with seq_lens[i] = 0 gives zeros; a row shorter than the prefix gives zeros and sets the
+ * STEP_ERR_INVALID_ARG bit of the device status word.  Only for pools the tensor-core kernel covers (bf16, head_dim
+ * 128, page_size 16, G <= 16) and n <= min(max_traces, 2048); otherwise STEP_ERR_INVALID_ARG, nothing launched. */
+int decode_attention_shared_prefix(step_pool* pool, int layer, const void* q,
+                                   const int32_t* block_table, const int32_t* seq_lens, int n,
+                                   const int32_t* prefix_blocks, int prefix_pages, void* out, void* stream);
+
 /* decode_attention without any caller-provided or allocated scratch.  (The paper has no
  * counterpart: this entry point exists for hosts, not for the method.)
  *

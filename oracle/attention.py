@@ -102,6 +102,34 @@ def paged_decode_attention(q: np.ndarray, k_pages: np.ndarray, v_pages: np.ndarr
     return out
 
 
+def paged_decode_attention_shared_prefix(q, k_pages, v_pages, block_table, seq_lens, prefix_blocks):
+    """Decode attention of traces whose first len(prefix_blocks) pages are the given shared blocks.
+
+    Trace t attends to the positions of the shared pages (in order) followed by its own positions
+    [len(prefix_blocks) * P, seq_lens[t]) read through its block-table row; this is paged_decode_attention whenever
+    the row's first entries equal prefix_blocks (the prompt pages all traces of one problem share: Algorithm 1,
+    InitTraces).  A trace with seq_lens[t] = 0, or shorter than the prefix, yields zeros; the ids of the latter are
+    returned as the second result.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    P = k_pages.shape[2]
+    pp = len(prefix_blocks)
+    out = np.zeros(q.shape, dtype=np.float64)
+    too_short = []
+    for t in range(q.shape[0]):
+        S = int(seq_lens[t])
+        if S == 0:
+            continue
+        if S < pp * P:
+            too_short.append(t)
+            continue
+        row = np.array(block_table[t]).copy()
+        row[:pp] = np.asarray(prefix_blocks)
+        K, V = gather_trace_kv(k_pages, v_pages, row, S)
+        out[t] = dense_decode_attention(q[t], K, V)
+    return out, too_short
+
+
 def merge_partials(ms, ls, os_):
     """Combine split evaluations of one softmax-weighted sum.
 

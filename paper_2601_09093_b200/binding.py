@@ -92,6 +92,7 @@ def lib():
     L.append_kv.argtypes = [vp, vp, i, i, vp, vp, vp]
     L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_static.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.decode_attention_shared_prefix.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
     L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
     L.score_steps_tokens.argtypes = [vp, vp, vp, vp, i, vp, i, C.POINTER(scorer_weights), vp, vp, vp]
     L.detect_step_ends.argtypes = [vp, vp, i, vp, i, vp, vp]
@@ -222,6 +223,15 @@ class KVPool:
             out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
         _check("decode_attention", lib().decode_attention(self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens),
                                                           n, _ptr(out), _stream(stream)))
+        return out
+
+    def decode_attention_shared_prefix(self, layer, q, block_table, seq_lens, prefix_blocks, prefix_pages, out=None, stream=None):
+        n = q.shape[0]
+        if out is None:
+            out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
+        _check("decode_attention_shared_prefix", lib().decode_attention_shared_prefix(
+            self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens), n, _ptr(prefix_blocks), prefix_pages,
+            _ptr(out), _stream(stream)))
         return out
 
     def decode_attention_static(self, layer, q, block_table, seq_lens, out, stream=None):

@@ -124,7 +124,18 @@ struct AttnArgs {
   int32_t* counters;
   int n, Hq, Hkv, G, max_pages, num_blocks;
   float scale_log2;
+  // shared-prefix passes only
+  const int32_t* prefix_blocks;    // [pp] block of every shared page
+  float* pre_ml;                   // [n][Hq][2]  (max, sum) of the attention over the shared pages, un-normalised
+  float* pre_o;                    // [n][Hq][kD] its weighted value sum
+  int pp;                          // shared pages
+  int tpb, n_bundles;              // prefix pass: traces per 16-row bundle of query rows, number of bundles
 };
+
+// kMode of attn_mma_kernel: the plain kernel; the pass over the shared pages, whose 16 query rows are the G heads of
+// tpb = 16 / G traces, so that one read of a shared page serves tpb traces, and which leaves (m, l, o) per
+// (trace, head) in pre_ml / pre_o; and the pass over every trace's own pages, which folds that result in at the end.
+constexpr int kPlain = 0, kPrefixPass = 1, kSuffixPass = 2;
 
 __device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -208,26 +219,39 @@ __device__ inline void cursor_next(Cursor& c, const int* cum, int n, int Hkv) {
   c.np = c.t < n ? cum[c.t + 1] - cum[c.t] : 1;
 }
 
-template <int kWarps, int kStages, bool kRows16>
+template <int kWarps, int kStages, bool kRows16, int kMode>
 __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
+  static_assert(kMode != kPrefixPass || kRows16, "the prefix pass uses all 16 rows of the tile");
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* s_pages = smem;                                              // [kWarps][kStages][8 KiB]
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kWarps * kStages * kPageBytes);
   int* s_cum = reinterpret_cast<int*>(s_bar + kWarps * kStages);              // [n + 1]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = a.n, Hkv = a.Hkv, G = a.G;
+  // n = sequences of the KV stream: traces, or (prefix pass) bundles of tpb traces that share the prefix pages
+  const int n = kMode == kPrefixPass ? a.n_bundles : a.n, Hkv = a.Hkv, G = a.G;
 
-  // ---- pages per trace, exclusive prefix sum (warp 0), barrier init (lane 0 of each warp)
+  // ---- pages per sequence, exclusive prefix sum (warp 0), barrier init (lane 0 of each warp)
   if (warp == 0) {
     int running = 0;
     for (int base = 0; base < n; base += 32) {
       const int t = base + lane;
       int pages = 0;
       if (t < n) {
-        int S = a.seq_lens[t];
-        if (S < 0) S = 0;
-        pages = (S + kP - 1) / kP;
-        if (pages > a.max_pages) { pages = a.max_pages; flag_error(a.counters, STEP_ERR_CAPACITY); }
+        if constexpr (kMode == kPrefixPass) {
+          // a bundle is read if one of its traces holds the whole prefix
+          for (int u = t * a.tpb; u < (t + 1) * a.tpb && u < a.n; ++u)
+            if (a.seq_lens[u] >= a.pp * kP) pages = a.pp;
+        } else {
+          int S = a.seq_lens[t];
+          if (S < 0) S = 0;
+          pages = (S + kP - 1) / kP;
+          if (pages > a.max_pages) { pages = a.max_pages; flag_error(a.counters, STEP_ERR_CAPACITY); }
+          if constexpr (kMode == kSuffixPass) {
+            // own pages only; a trace shorter than the prefix it is said to share is flagged and gets zeros
+            if (S >= a.pp * kP) pages -= a.pp;
+            else { pages = 0; if (S > 0) flag_error(a.counters, STEP_ERR_INVALID_ARG); }
+          }
+        }
       }
       int incl = pages;
 #pragma unroll
@@ -247,10 +271,19 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   }
   __syncthreads();
 
-  // traces without any position get zeros (CTAs take the traces round-robin)
-  for (int t = blockIdx.x; t < n; t += gridDim.x)
-    if (s_cum[t + 1] == s_cum[t])
-      for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) a.out[(size_t)t * a.Hq * kD + k] = 0.f;
+  // traces without any position get zeros (CTAs take the traces round-robin); in the suffix pass a trace that
+  // holds the prefix and nothing else gets the normalised prefix result
+  if constexpr (kMode != kPrefixPass) {
+    for (int t = blockIdx.x; t < n; t += gridDim.x)
+      if (s_cum[t + 1] == s_cum[t]) {
+        const bool prefix_only = kMode == kSuffixPass && a.seq_lens[t] >= a.pp * kP;
+        for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) {
+          float v = 0.f;
+          if (prefix_only) v = a.pre_o[(size_t)t * a.Hq * kD + k] / a.pre_ml[((size_t)t * a.Hq + k / kD) * 2 + 1];
+          a.out[(size_t)t * a.Hq * kD + k] = v;
+        }
+      }
+  }
 
   const long long total = (long long)Hkv * s_cum[n];
   const int n_part = gridDim.x * kWarps;
@@ -273,7 +306,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     if (pc.t != win_t || pc.page < win_base || pc.page >= win_base + 32) {
       win_t = pc.t; win_base = pc.page;
       const int pg = win_base + lane;
-      win_ids = pg < pc.np ? a.block_table[(size_t)pc.t * a.max_pages + pg] : 0;
+      if constexpr (kMode == kPrefixPass) win_ids = pg < pc.np ? a.prefix_blocks[pg] : 0;
+      else if constexpr (kMode == kSuffixPass) win_ids = pg < pc.np ? a.block_table[(size_t)pc.t * a.max_pages + a.pp + pg] : 0;
+      else win_ids = pg < pc.np ? a.block_table[(size_t)pc.t * a.max_pages + pg] : 0;
     }
     int b = __shfl_sync(0xffffffffu, win_ids, pc.page - win_base);
     if (lane == 0) {
@@ -311,10 +346,21 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   for (int i = 0; i < cnt; ++i) {
     if (!seg_open) {
       // new (trace, head) segment: Q fragments of the G heads of this group, fresh softmax state
-      const __nv_bfloat16* qbase = a.q + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
-      const uint32_t* q0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)g_row * kD);
-      const uint32_t* q1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(g_row + 8) * kD);
-      const bool r0 = g_row < G, r1 = kRows16 && (g_row + 8 < G);
+      const uint32_t *q0, *q1;
+      bool r0, r1;
+      if constexpr (kMode == kPrefixPass) {
+        // row r of the tile is head (r % G) of the group of trace cc.t * tpb + r / G
+        const int ta = cc.t * a.tpb + g_row / G, tb = cc.t * a.tpb + (g_row + 8) / G;
+        r0 = g_row < a.tpb * G && ta < a.n;
+        r1 = g_row + 8 < a.tpb * G && tb < a.n;
+        q0 = reinterpret_cast<const uint32_t*>(a.q + ((size_t)(r0 ? ta : 0) * a.Hq + (size_t)cc.h * G + g_row % G) * kD);
+        q1 = reinterpret_cast<const uint32_t*>(a.q + ((size_t)(r1 ? tb : 0) * a.Hq + (size_t)cc.h * G + (g_row + 8) % G) * kD);
+      } else {
+        const __nv_bfloat16* qbase = a.q + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
+        q0 = reinterpret_cast<const uint32_t*>(qbase + (size_t)g_row * kD);
+        q1 = reinterpret_cast<const uint32_t*>(qbase + (size_t)(g_row + 8) * kD);
+        r0 = g_row < G; r1 = kRows16 && (g_row + 8 < G);
+      }
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         qa[ks][0] = r0 ? q0[ks * 8 + tq] : 0u;
@@ -340,11 +386,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
     // tokens of this page that exist (only the last page of a sequence can be short)
     int valid = kP;
-    if (cc.page == cc.np - 1) {
+    if (kMode != kPrefixPass && cc.page == cc.np - 1) {    // shared pages are full
       int S = a.seq_lens[cc.t];
       const int cap = a.max_pages * kP;
       if (S > cap) S = cap;
-      valid = S - cc.page * kP;
+      valid = S - (cc.page + (kMode == kSuffixPass ? a.pp : 0)) * kP;
       if (valid < kP) {
         // unused V rows may hold anything (even NaN bit patterns): zero them so 0 * V stays 0
         for (int idx = lane; idx < (kP - valid) * 16; idx += 32) {
@@ -433,31 +479,81 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
       }
       const bool complete = seg_first_page == 0 && cc.page + 1 == cc.np;
-      if (complete) {
+      const int R = kMode == kPrefixPass ? 16 : G;       // rows of a partial slot
+      if (complete && kMode == kPrefixPass) {
+        // the bundle's whole prefix was read by this warp: (m, l, o) of every (trace, head) row, un-normalised
+        const int ta = cc.t * a.tpb + g_row / G, tb = cc.t * a.tpb + (g_row + 8) / G;
+        if (g_row < a.tpb * G && ta < a.n) {
+          const size_t idx = (size_t)ta * a.Hq + (size_t)cc.h * G + g_row % G;
+          if (tq == 0) { a.pre_ml[idx * 2] = m_run[0]; a.pre_ml[idx * 2 + 1] = l0; }
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(a.pre_o + idx * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][0], o_acc[dt][1]);
+        }
+        if (g_row + 8 < a.tpb * G && tb < a.n) {
+          const size_t idx = (size_t)tb * a.Hq + (size_t)cc.h * G + (g_row + 8) % G;
+          if (tq == 0) { a.pre_ml[idx * 2] = m_run[1]; a.pre_ml[idx * 2 + 1] = l1; }
+#pragma unroll
+          for (int dt = 0; dt < 16; ++dt)
+            *reinterpret_cast<float2*>(a.pre_o + idx * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2], o_acc[dt][3]);
+        }
+      } else if (complete) {
         float* ob = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
         if (g_row < G) {
-          const float inv = 1.f / l0;
+          float ws = 1.f, wp = 0.f, lp = 0.f;
+          const float* po = nullptr;
+          if constexpr (kMode == kSuffixPass) {          // fold in the shared pages' result
+            const size_t idx = (size_t)cc.t * a.Hq + (size_t)cc.h * G + g_row;
+            const float mp = a.pre_ml[idx * 2];
+            lp = a.pre_ml[idx * 2 + 1];
+            const float Mn = fmaxf(m_run[0], mp);
+            ws = exp2f(m_run[0] - Mn); wp = exp2f(mp - Mn);
+            po = a.pre_o + idx * kD;
+          }
+          const float inv = 1.f / (l0 * ws + lp * wp);
 #pragma unroll
-          for (int dt = 0; dt < 16; ++dt)
-            *reinterpret_cast<float2*>(ob + (size_t)g_row * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][0] * inv, o_acc[dt][1] * inv);
+          for (int dt = 0; dt < 16; ++dt) {
+            float x = o_acc[dt][0] * ws, y = o_acc[dt][1] * ws;
+            if constexpr (kMode == kSuffixPass) {
+              const float2 pv = *reinterpret_cast<const float2*>(po + dt * 8 + 2 * tq);
+              x += wp * pv.x; y += wp * pv.y;
+            }
+            *reinterpret_cast<float2*>(ob + (size_t)g_row * kD + dt * 8 + 2 * tq) = make_float2(x * inv, y * inv);
+          }
         }
         if (kRows16 && g_row + 8 < G) {
-          const float inv = 1.f / l1;
+          float ws = 1.f, wp = 0.f, lp = 0.f;
+          const float* po = nullptr;
+          if constexpr (kMode == kSuffixPass) {
+            const size_t idx = (size_t)cc.t * a.Hq + (size_t)cc.h * G + g_row + 8;
+            const float mp = a.pre_ml[idx * 2];
+            lp = a.pre_ml[idx * 2 + 1];
+            const float Mn = fmaxf(m_run[1], mp);
+            ws = exp2f(m_run[1] - Mn); wp = exp2f(mp - Mn);
+            po = a.pre_o + idx * kD;
+          }
+          const float inv = 1.f / (l1 * ws + lp * wp);
 #pragma unroll
-          for (int dt = 0; dt < 16; ++dt)
-            *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2] * inv, o_acc[dt][3] * inv);
+          for (int dt = 0; dt < 16; ++dt) {
+            float x = o_acc[dt][2] * ws, y = o_acc[dt][3] * ws;
+            if constexpr (kMode == kSuffixPass) {
+              const float2 pv = *reinterpret_cast<const float2*>(po + dt * 8 + 2 * tq);
+              x += wp * pv.x; y += wp * pv.y;
+            }
+            *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(x * inv, y * inv);
+          }
         }
       } else {
         const size_t slot = (size_t)part * 2 + (seg_is_first ? 0 : 1);
-        float* ml = a.ws_ml + slot * G * 2;
-        float* ob = a.ws_o + slot * G * kD;
-        if (g_row < G) {
+        float* ml = a.ws_ml + slot * R * 2;
+        float* ob = a.ws_o + slot * R * kD;
+        if (g_row < R) {
           if (tq == 0) { ml[g_row * 2] = m_run[0]; ml[g_row * 2 + 1] = l0; }
 #pragma unroll
           for (int dt = 0; dt < 16; ++dt)
             *reinterpret_cast<float2*>(ob + (size_t)g_row * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][0], o_acc[dt][1]);
         }
-        if (kRows16 && g_row + 8 < G) {
+        if (kRows16 && g_row + 8 < R) {
           if (tq == 0) { ml[(g_row + 8) * 2] = m_run[1]; ml[(g_row + 8) * 2 + 1] = l1; }
 #pragma unroll
           for (int dt = 0; dt < 16; ++dt)
@@ -474,24 +570,44 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
         if (ticket == w_last - w_first) {
           if (lane == 0) a.seg_cnt[cc.t * Hkv + cc.h] = 0;             // ready for the next launch
           __threadfence();
-          float* og = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
-          for (int g = 0; g < G; ++g) {
-            float M = -INFINITY;
+          const int rows = kMode == kPrefixPass ? a.tpb * G : G;
+          for (int g = 0; g < rows; ++g) {
+            size_t idx = 0;                                            // (trace, head) row of pre_ml / pre_o
+            if constexpr (kMode == kPrefixPass) {
+              const int t = cc.t * a.tpb + g / G;
+              if (t >= a.n) break;
+              idx = (size_t)t * a.Hq + (size_t)cc.h * G + g % G;
+            } else if constexpr (kMode == kSuffixPass) {
+              idx = (size_t)cc.t * a.Hq + (size_t)cc.h * G + g;
+            }
+            float M = kMode == kSuffixPass ? a.pre_ml[idx * 2] : -INFINITY;
             for (int w = w_first; w <= w_last; ++w) {
               const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
-              M = fmaxf(M, __ldcg(&a.ws_ml[(sl * G + g) * 2]));
+              M = fmaxf(M, __ldcg(&a.ws_ml[(sl * R + g) * 2]));
             }
             float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
             float den = 0.f;
+            if constexpr (kMode == kSuffixPass) {                      // the shared pages count as one more partial
+              const float wgt = exp2f(a.pre_ml[idx * 2] - M);
+              den = wgt * a.pre_ml[idx * 2 + 1];
+              const float4 o4 = reinterpret_cast<const float4*>(a.pre_o + idx * kD)[lane];
+              num = make_float4(wgt * o4.x, wgt * o4.y, wgt * o4.z, wgt * o4.w);
+            }
             for (int w = w_first; w <= w_last; ++w) {
               const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
-              const float wgt = exp2f(__ldcg(&a.ws_ml[(sl * G + g) * 2]) - M);
-              den += wgt * __ldcg(&a.ws_ml[(sl * G + g) * 2 + 1]);
-              const float4 o4 = __ldcg(reinterpret_cast<const float4*>(a.ws_o + (sl * G + g) * kD) + lane);
+              const float wgt = exp2f(__ldcg(&a.ws_ml[(sl * R + g) * 2]) - M);
+              den += wgt * __ldcg(&a.ws_ml[(sl * R + g) * 2 + 1]);
+              const float4 o4 = __ldcg(reinterpret_cast<const float4*>(a.ws_o + (sl * R + g) * kD) + lane);
               num.x += wgt * o4.x; num.y += wgt * o4.y; num.z += wgt * o4.z; num.w += wgt * o4.w;
             }
-            const float inv = 1.f / den;
-            reinterpret_cast<float4*>(og + (size_t)g * kD)[lane] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+            if constexpr (kMode == kPrefixPass) {
+              if (lane == 0) { a.pre_ml[idx * 2] = M; a.pre_ml[idx * 2 + 1] = den; }
+              reinterpret_cast<float4*>(a.pre_o + idx * kD)[lane] = num;
+            } else {
+              float* og = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
+              const float inv = 1.f / den;
+              reinterpret_cast<float4*>(og + (size_t)g * kD)[lane] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+            }
           }
         }
       }
@@ -514,22 +630,36 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
 constexpr int kWarpsDefault = 8, kStagesDefault = 3;
 
-template <int kWarps, int kStages>
-int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s) {
+template <int kWarps, int kStages, bool kRows16, int kMode>
+int launch_one(const AttnArgs& a, int grid, cudaStream_t s) {
   const size_t smem = (size_t)kWarps * kStages * kPageBytes + (size_t)kWarps * kStages * 8 + (size_t)(a.n + 1) * 4;
+  auto kern = attn_mma_kernel<kWarps, kStages, kRows16, kMode>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+  kern<<<grid, kWarps * 32, smem, s>>>(a);
+  return launch_ok();
+}
+
+template <int kWarps, int kStages, int kMode>
+int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s) {
   int grid = pool->attn_grid;
   if (grid * kWarps > kMaxPartitions) grid = kMaxPartitions / kWarps;
   if (grid < 1) grid = 1;
-  if (a.G > 8) {
-    auto kern = attn_mma_kernel<kWarps, kStages, true>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
-    kern<<<grid, kWarps * 32, smem, s>>>(a);
-  } else {
-    auto kern = attn_mma_kernel<kWarps, kStages, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
-    kern<<<grid, kWarps * 32, smem, s>>>(a);
-  }
-  return launch_ok();
+  return a.G > 8 ? launch_one<kWarps, kStages, true, kMode>(a, grid, s) : launch_one<kWarps, kStages, false, kMode>(a, grid, s);
+}
+
+void fill_args(AttnArgs& a, const step_pool* pool, const Geo& g, int layer, const void* q, const int32_t* block_table,
+               const int32_t* seq_lens, int n, void* out) {
+  a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
+  a.q = (const __nv_bfloat16*)q;
+  a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
+  a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.seg_cnt = pool->v.attn_cnt; a.counters = pool->v.counters;
+  a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
+  a.prefix_blocks = nullptr; a.pre_ml = nullptr; a.pre_o = nullptr; a.pp = 0; a.tpb = 1; a.n_bundles = 0;
+}
+
+bool mma_shape(const step_pool* pool, const Geo& g, int n) {
+  return pool->cfg.dtype == STEP_BF16 && g.d == kD && g.P == kP && g.G <= 16 && n <= kMaxTracesFast && pool->swizzle;
 }
 
 }  // namespace
@@ -542,17 +672,10 @@ extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const
   Geo g = geo_of(pool);
   if (layer < 0 || layer >= g.L) return STEP_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  const bool fast = pool->fast_path > 0 && pool->cfg.dtype == STEP_BF16 && g.d == kD && g.P == kP &&
-                    g.G <= 16 && n <= kMaxTracesFast && pool->swizzle;
-  if (fast) {
+  if (pool->fast_path > 0 && mma_shape(pool, g, n)) {
     AttnArgs a;
-    a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
-    a.q = (const __nv_bfloat16*)q;
-    a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
-    a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.seg_cnt = pool->v.attn_cnt; a.counters = pool->v.counters;
-    a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
-    a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
-    return launch_mma<kWarpsDefault, kStagesDefault>(pool, a, s);
+    fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
+    return launch_mma<kWarpsDefault, kStagesDefault, kPlain>(pool, a, s);
   }
   if (n > 65535) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)(g.d + kScalarWarps * g.d) * sizeof(float);
@@ -565,6 +688,41 @@ extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const
         g, (const float*)pool->cfg.kv_storage, layer, (const float*)q, block_table, seq_lens, (float*)out,
         pool->v.counters);
   return launch_ok();
+}
+
+// decode_attention when the first prefix_pages pages of every listed trace are the same blocks (the prompt pages
+// kv_pool_fork_prefix shares between the traces of one problem).  Two launches: the shared pages are read once per
+// bundle of 16 / G traces instead of once per trace, then every trace's own pages are read as usual and the two
+// results combined by the usual (max, sum) rule.  HBM traffic is the same as decode_attention's (the L2 absorbs
+// the repeated reads there); what shrinks is the L2 -> SM traffic, which is what bounds the step when the prompt
+// is long against the generated suffixes.
+extern "C" int decode_attention_shared_prefix(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                              const int32_t* seq_lens, int n, const int32_t* prefix_blocks,
+                                              int prefix_pages, void* out, void* stream) {
+  if (!pool || n < 0 || prefix_pages < 0) return STEP_ERR_INVALID_ARG;
+  if (prefix_pages == 0) return decode_attention(pool, layer, q, block_table, seq_lens, n, out, stream);
+  if (n == 0) return STEP_OK;
+  if (!q || !block_table || !seq_lens || !out || !prefix_blocks) return STEP_ERR_INVALID_ARG;
+  Geo g = geo_of(pool);
+  if (layer < 0 || layer >= g.L || prefix_pages > g.max_pages) return STEP_ERR_INVALID_ARG;
+  if (!mma_shape(pool, g, n) || n > g.max_traces || !pool->v.pre_o) return STEP_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  AttnArgs a;
+  fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
+  a.prefix_blocks = prefix_blocks; a.pre_ml = pool->v.pre_ml; a.pre_o = pool->v.pre_o; a.pp = prefix_pages;
+  a.tpb = 16 / g.G; a.n_bundles = (n + a.tpb - 1) / a.tpb;
+  // pass 1: about eight pages per warp, at most one CTA per SM and kPrefixPartitions partitions
+  AttnArgs p1 = a;
+  p1.ws_ml = pool->v.pre_ws_ml; p1.ws_o = pool->v.pre_ws_o;
+  const long long pages1 = (long long)a.n_bundles * g.Hkv * prefix_pages;
+  long long grid1 = (pages1 + kWarpsDefault * 8 - 1) / (kWarpsDefault * 8);
+  const int cap1 = pool->attn_grid < kPrefixPartitions / kWarpsDefault ? pool->attn_grid : kPrefixPartitions / kWarpsDefault;
+  if (grid1 > cap1) grid1 = cap1;
+  if (grid1 < 1) grid1 = 1;
+  const int st = launch_one<kWarpsDefault, kStagesDefault, true, kPrefixPass>(p1, (int)grid1, s);
+  if (st != STEP_OK) return st;
+  // pass 2
+  return launch_mma<kWarpsDefault, kStagesDefault, kSuffixPass>(pool, a, s);
 }
 
 // =============================================================== allocation-free variant
@@ -642,7 +800,7 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
   const size_t smem = (size_t)kWarpsDefault * kStagesDefault * kPageBytes + (size_t)kWarpsDefault * kStagesDefault * 8 +
                       (size_t)(n + 1) * 4;
-  auto kern = attn_mma_kernel<kWarpsDefault, kStagesDefault, false>;
+  auto kern = attn_mma_kernel<kWarpsDefault, kStagesDefault, false, kPlain>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
   cudaStream_t s = (cudaStream_t)stream;
   kern<<<grid, kWarpsDefault * 32, smem, s>>>(a);

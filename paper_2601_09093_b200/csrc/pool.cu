@@ -53,6 +53,12 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
   l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
   l.attn_cnt = take((size_t)kMaxTracesFast * c->num_kv_heads * 4);
+  // shared-prefix attention: partials of its first pass (16 query rows per slot) and that pass's result per (trace, head)
+  const bool mma = c->dtype == STEP_BF16 && c->head_dim == 128 && c->page_size == 16;
+  l.pre_ws_ml = take(mma ? (size_t)kPrefixPartitions * 2 * 16 * 2 * 4 : 0);
+  l.pre_ws_o = take(mma ? (size_t)kPrefixPartitions * 2 * 16 * c->head_dim * 4 : 0);
+  l.pre_ml = take(mma ? T * c->num_q_heads * 2 * 4 : 0);
+  l.pre_o = take(mma ? T * c->num_q_heads * c->head_dim * 4 : 0);
   l.final_score = take(T * 4);
   l.answer = take(T * 4);
   l.finished = take(T);
@@ -328,6 +334,9 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
   v.score_part = (float2*)(m + lay.score_part);
   v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o); v.attn_cnt = (int32_t*)(m + lay.attn_cnt);
+  const bool mma = lay.pre_ws_o != lay.pre_ml;      // the regions are zero-sized for other shapes
+  v.pre_ws_ml = mma ? (float*)(m + lay.pre_ws_ml) : nullptr; v.pre_ws_o = mma ? (float*)(m + lay.pre_ws_o) : nullptr;
+  v.pre_ml = mma ? (float*)(m + lay.pre_ml) : nullptr; v.pre_o = mma ? (float*)(m + lay.pre_o) : nullptr;
   v.final_score = (float*)(m + lay.final_score); v.answer = (int32_t*)(m + lay.answer);
   v.finished = (uint8_t*)(m + lay.finished); v.it_ids = (int32_t*)(m + lay.it_ids);
   v.it_fin = (int32_t*)(m + lay.it_fin); v.it_pruned = (int32_t*)(m + lay.it_pruned);

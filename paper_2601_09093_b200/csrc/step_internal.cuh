@@ -20,6 +20,7 @@
 namespace stepk {
 
 constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream partitions of one launch
+constexpr int kPrefixPartitions = 1184; // partitions of the shared-prefix pass of decode_attention_shared_prefix (148 SMs x 8 warps)
 constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
 constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
 constexpr int kScoreFoldRows = 512;    // listed rows one CTA of the scorer's finishing kernel folds into per-trace partials
@@ -40,6 +41,7 @@ struct MetaLayout {
   size_t append_base, prune_rank, prune_list, prune_off;
   size_t score_idx, score_z, score_part;
   size_t attn_ml, attn_o, attn_cnt;
+  size_t pre_ws_ml, pre_ws_o, pre_ml, pre_o;   // shared-prefix attention (zero-sized for pools the tensor-core kernel does not cover)
   size_t final_score, answer, finished, it_ids, it_fin, it_pruned;
   size_t total;
 };
@@ -51,6 +53,7 @@ struct DevViews {
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
   int32_t* score_idx; float* score_z; float2* score_part;
   float* attn_ml; float* attn_o; int32_t* attn_cnt;
+  float* pre_ws_ml; float* pre_ws_o; float* pre_ml; float* pre_o;   // null when zero-sized
   float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
   int32_t* it_ids; int32_t* it_fin; int32_t* it_pruned;       // per-iteration lists of the Algorithm 1 driver
 };

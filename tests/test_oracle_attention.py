@@ -143,3 +143,38 @@ def test_large_logits_do_not_overflow():
 
 def test_flop_count():
     assert A.attention_flops(32, 128, 1000) == 4 * 32 * 128 * 1000
+
+
+def test_shared_prefix_attention_definition():
+    """With shared first pages it is the plain paged attention; with rows that do not share them it is dense attention
+    over (shared pages ++ own positions) assembled by hand; short and empty rows give zeros."""
+    g = np.random.default_rng(21)
+    NB, Hkv, P, d, Hq = 20, 2, 4, 8, 4
+    kp, vp = g.standard_normal((NB, Hkv, P, d)), g.standard_normal((NB, Hkv, P, d))
+    q = g.standard_normal((4, Hq, d))
+    shared = [7, 3]
+    bt = np.full((4, 5), -1)
+    bt[0, :4] = [7, 3, 10, 11]; bt[1, :3] = [7, 3, 12]; bt[2, :2] = [7, 3]; bt[3, :3] = [7, 3, 13]
+    sl = np.array([14, 9, 8, 0])
+    want = A.paged_decode_attention(q, kp, vp, bt, sl)
+    got, short = A.paged_decode_attention_shared_prefix(q, kp, vp, bt, sl, shared)
+    assert short == []
+    np.testing.assert_array_equal(got, want)
+    assert np.all(got[3] == 0)
+    # rows whose own first pages differ: the shared blocks are used all the same
+    bt2 = bt.copy(); bt2[0, :2] = [1, 2]; bt2[1, :2] = [-1, -1]
+    got2, _ = A.paged_decode_attention_shared_prefix(q, kp, vp, bt2, sl, shared)
+    np.testing.assert_array_equal(got2, want)
+    # by hand for trace 0: 8 shared positions, then blocks 10 and 11 (6 of their 8 slots)
+    K = np.concatenate([kp[7].swapaxes(0, 1), kp[3].swapaxes(0, 1), kp[10].swapaxes(0, 1), kp[11].swapaxes(0, 1)[:2]])
+    V = np.concatenate([vp[7].swapaxes(0, 1), vp[3].swapaxes(0, 1), vp[10].swapaxes(0, 1), vp[11].swapaxes(0, 1)[:2]])
+    np.testing.assert_allclose(got[0], A.dense_decode_attention(q[0], K, V), rtol=0, atol=1e-15)
+    # a row shorter than the prefix
+    sl3 = np.array([14, 5, 8, 0])
+    got3, short3 = A.paged_decode_attention_shared_prefix(q, kp, vp, bt, sl3, shared)
+    assert short3 == [1] and np.all(got3[1] == 0)
+    np.testing.assert_array_equal(got3[0], want[0])
+    # split identity: prefix partial merged with the suffix partial is the whole
+    Kg, Vg = K[:, 0], V[:, 0]
+    parts = [A.partial_of_range(q[0, 1], Kg, Vg, 0, 8), A.partial_of_range(q[0, 1], Kg, Vg, 8, 14)]
+    np.testing.assert_allclose(A.merge_partials(*zip(*parts)), got[0, 1], rtol=0, atol=1e-14)
