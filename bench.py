@@ -38,7 +38,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer", "prefix"])
+    ap.add_argument("--prefix-len", type=int, default=8192, help="prefix workload: tokens of the shared prompt")
+    ap.add_argument("--suffix-max", type=int, default=512, help="prefix workload: traces hold 1 .. this many tokens of their own")
     ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
     ap.add_argument("--scorer-density", type=float, default=1.0, help="fraction of those rows that end a step")
     ap.add_argument("--scorer-shape", default="c1", choices=["c1", "c4"])
@@ -706,6 +708,75 @@ def run_scorer(args):
 
 
 # ---------------------------------------------------------------------------------------------
+def run_prefix(args):
+    """`--workload prefix`: decode_attention and decode_attention_shared_prefix on the same state - 64 traces of the
+    8B layout whose shared prompt is long against what each trace generated (the regime the paper's workloads are
+    NOT in: there the prompt is a few hundred tokens of tens of thousands).  One layer; single GPU."""
+    import torch
+    from paper_2601_09093_b200 import binding as B, harness as H, ranks as R, workloads as W
+    from paper_2601_09093_b200 import build as _build
+    rank, local_rank, world = R.rank_env()
+    if rank != 0:
+        return
+    _build.build()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    B.lib()
+    cfg = W.scaled(W.C1, name="prefix-heavy-1layer", prefix_len=args.prefix_len, suffix_lo=1, suffix_hi=args.suffix_max)
+    T, P = cfg.n_traces, cfg.page_size
+    suffix = W.suffix_lengths(cfg)
+    pp = cfg.prefix_len // P
+    pages = pp + int(sum(-(-(cfg.prefix_len % P + int(x)) // P) for x in suffix))
+    pool = H.make_pool(cfg, pages + 64, -(-(cfg.prefix_len + int(suffix.max())) // P) + 2, T, device=dev)
+    H.fill_random_device(pool, cfg, suffix, seed=cfg.seed)
+    v = pool.views()
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 1)
+    q = torch.randn((T, cfg.num_q_heads, cfg.head_dim), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out_a = torch.empty((T, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
+    out_b = torch.empty_like(out_a)
+    prefix_blocks = v["block_table"][0, :pp].contiguous()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    K, Wm = max(args.steps, 3), max(args.warmup, 3)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        ts = []
+        for i in range(Wm + K):
+            flush.zero_()                                          # L2 flush: the state itself is smaller than L2
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); fn(); e1.record(stream)
+            torch.cuda.synchronize()
+            if i >= Wm:
+                ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    sampler = ClockSampler(local_rank); sampler.start()
+    ms_plain = timed(lambda: pool.decode_attention(0, q, v["block_table"], v["seq_lens"], out_a))
+    ms_shared = timed(lambda: pool.decode_attention_shared_prefix(0, q, v["block_table"], v["seq_lens"], prefix_blocks, pp, out_b))
+    clocks = sampler.stop()
+    err_code, err_mask = pool.last_error()
+    logical = float(T * cfg.prefix_len + suffix.sum()) * cfg.bytes_per_token_layer
+    unique = H.unique_kv_bytes(cfg, cfg.prefix_len, suffix)
+    peak, peak_kind = measured_peaks()
+    res = {"metric": "trace-layer decode steps/s (one layer, shared-prefix attention)", "value": T / (ms_shared * 1e-3),
+           "unit": "trace-layer-steps/s", "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": ms_shared,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic (seeded, drawn on device)",
+           "config": {"workload": cfg.name, "traces": T, "prefix_len": cfg.prefix_len, "suffix": "1..%d" % args.suffix_max,
+                      "shared_pages": pp, "l2_policy": "L2 flushed (256 MB written) before every timed launch"},
+           "plain": {"ms": ms_plain, "logical_gbs": logical / ms_plain / 1e6, "unique_gbs": unique / ms_plain / 1e6},
+           "shared_prefix": {"ms": ms_shared, "logical_gbs": logical / ms_shared / 1e6, "unique_gbs": unique / ms_shared / 1e6,
+                             "launches": 2},
+           "speedup": ms_plain / ms_shared, "max_abs_diff": float((out_a - out_b).abs().max()),
+           "roofline": {"bound": "hbm", "achieved": unique / ms_shared / 1e6, "peak": peak, "unit": "GB/s",
+                        "frac": unique / ms_shared / 1e6 / peak, "peak_kind": "of " + peak_kind, "traffic": None,
+                        "kernel": "decode_attention_shared_prefix (two launches of attn_mma_kernel)",
+                        "note": "a %.0f MB launch: fixed launch costs weigh on it" % (unique / 1e6)},
+           "gpu_launches": 3 * K, "clocks": clocks, "status": {"device_error_mask": err_mask}}
+    print(json.dumps(res))
+
+
+# ---------------------------------------------------------------------------------------------
 def run_reference(args):
     """The reference arm is the CPU oracle, as it stands, on the host cores.
     Under a multi-rank launcher rank 0 alone runs and prints; the other ranks leave at once."""
@@ -804,8 +875,12 @@ def run_reference_scorer(args, K, Wm, sample=64):
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
+        if a.workload == "prefix":
+            a.workload = "c1"           # the oracle's arm of the prefix workload is the one-layer configuration it is cut from
         run_reference(a)
     elif a.workload == "scorer":
         run_scorer(a)
+    elif a.workload == "prefix":
+        run_prefix(a)
     else:
         run_ours(a)
