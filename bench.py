@@ -172,7 +172,7 @@ def run_ours(args):
 
     K, Wm = args.steps, max(args.warmup, 3)
     e2e_steps = 0 if args.no_e2e else K
-    steps_total = Wm + K + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS + 3
+    steps_total = Wm + K + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS + 3 + ALG1_GRAPH_ITERATIONS + 2
     free_b, total_b = torch.cuda.mem_get_info(dev)
     cfg, suffix, nb, max_pages, phys_layers = workload_plan(args.workload, args.num_blocks, steps_total, free_b,
                                                             args.traces, args.threshold)
@@ -441,6 +441,7 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
 
 # ---------------------------------------------------------------------------------------------
 ALG1_ITERATIONS = 6
+ALG1_GRAPH_ITERATIONS = 40          # iterations of the recorded-iteration run on the one-layer workloads (6 on the others)
 
 
 def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host, ms_per_step_python):
@@ -454,7 +455,7 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     table = B.step_end_table_from_vocab(vocab)
     ends = np.flatnonzero(table.numpy())
     toks = np.stack([W.token_ids(cfg.seed, T, len(vocab), ends, cfg.boundary_density, sub=500 + i)
-                     for i in range(ALG1_ITERATIONS + 2)])
+                     for i in range(ALG1_ITERATIONS + 2 + ALG1_GRAPH_ITERATIONS + 2)])
     toks[toks == 0] = 1                                            # id 0 is the end-of-sequence token here: nobody completes
     table_d, toks_d = table.to(dev), torch.from_numpy(toks).to(dev)
     q = torch.stack([s["q"][:phys_layers] for s in sets]).contiguous()
@@ -464,9 +465,9 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     answers = torch.zeros(T, dtype=torch.int32, device=dev)
     attn_out = torch.empty((phys_layers, T, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device=dev)
 
-    def run(tok, n):
+    def run(tok, n, graphs=False):
         r = pool.algorithm1_run(tok, 0, table_d, answers, q, k, v, h, wts, cfg.threshold, cfg.keep_frac,
-                                check_every=n, attn_out=attn_out)
+                                check_every=n, attn_out=attn_out, use_graphs=graphs)
         for _ in range(n):
             append_log.append((ids_host, 1))
         return r
@@ -474,10 +475,25 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     run(toks_d[:2], 2)                                              # warm-up
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    r = run(toks_d[2:], ALG1_ITERATIONS)
+    r = run(toks_d[2:2 + ALG1_ITERATIONS], ALG1_ITERATIONS)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / ALG1_ITERATIONS
+    # the same loop with each ring slot's iteration recorded as a CUDA graph (on a stream that can be captured); the
+    # timed call records its two graphs itself, so that cost is inside the figure
+    n_g = ALG1_GRAPH_ITERATIONS if phys_layers == 1 else 6
+    base = 2 + ALG1_ITERATIONS
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run(toks_d[base:base + 2], 2, graphs=True)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(side)
+        rg = run(toks_d[base + 2:base + 2 + n_g], n_g, graphs=True)
+        g1.record(side)
+    torch.cuda.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    ms_g = g0.elapsed_time(g1) / n_g
     # step-end detection alone
     n_tok = 1 << 22
     big = torch.from_numpy(W.token_ids(cfg.seed, n_tok, len(vocab), ends, cfg.boundary_density, sub=77)).to(dev)
@@ -496,6 +512,9 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
             "vs_python_driven_step": None if ms_per_step_python is None else ms_per_step_python / ms,
             "layers_per_iteration": phys_layers, "launches_per_iteration": 8 + phys_layers,
             "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
+            "recorded_iterations": {"iterations": rg["iterations"], "ms_per_iteration": ms_g,
+                                    "trace_decode_steps_per_s": T / (ms_g * 1e-3), "vs_direct_launches": ms / ms_g,
+                                    "live_left": rg["live_left"]},
             "detect_step_ends": {"tokens": n_tok, "us_per_call": det_ms * 1e3, "tokens_per_s": n_tok / (det_ms * 1e-3),
                                  "gbs": n_tok * 5 / (det_ms * 1e-3) / 1e9},
             "device_error_mask": bits}

@@ -279,6 +279,11 @@ typedef struct {
   int max_evictions;                  /* as in step_iteration                                                     */
   int check_every;                    /* the host asks for the number of live traces every this many iterations   */
   float* score_history;               /* [max_iterations, n] score_t after each iteration's scoring, or NULL      */
+  int use_graphs;                     /* != 0: the launches of one iteration are recorded once per ring slot as a CUDA
+                                         graph and replayed (one graph launch per iteration instead of a dozen kernel
+                                         launches; worth it when an iteration is short).  Needs a stream that can be
+                                         captured (not the default stream, not already capturing), else ignored.  The
+                                         graphs are private to the call and destroyed before it returns.              */
 } step_run_args;
 
 typedef struct {

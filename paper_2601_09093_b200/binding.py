@@ -57,7 +57,8 @@ class step_run_args(C.Structure):
                 ("n_layers_attention", C.c_int), ("q", C.c_void_p), ("k_new", C.c_void_p), ("v_new", C.c_void_p),
                 ("hidden", C.c_void_p), ("attn_out", C.c_void_p), ("step_scores_out", C.c_void_p),
                 ("scorer", C.POINTER(scorer_weights)), ("threshold", C.c_float), ("keep_frac", C.c_float),
-                ("max_evictions", C.c_int), ("check_every", C.c_int), ("score_history", C.c_void_p)]
+                ("max_evictions", C.c_int), ("check_every", C.c_int), ("score_history", C.c_void_p),
+                ("use_graphs", C.c_int)]
 
 
 class step_run_result(C.Structure):
@@ -336,7 +337,8 @@ class KVPool:
         return attn_out, step_scores_out
 
     def algorithm1_run(self, token_ids, eos_token, step_end_table, answers, q, k_new, v_new, hidden, weights, threshold,
-                       keep_frac, max_evictions=1, check_every=16, attn_out=None, score_history=None, stream=None):
+                       keep_frac, max_evictions=1, check_every=16, attn_out=None, score_history=None, stream=None,
+                       use_graphs=False):
         """The whole loop.  token_ids: [max_iterations, n]; q: [ring, layers, n, Hq, d] or None;
         k_new, v_new: [ring, n, 1, L, Hkv, d]; hidden: [ring, n, D].  Returns the result as a dict (synchronises)."""
         max_it, n = token_ids.shape
@@ -350,7 +352,7 @@ class KVPool:
                           ring=ring, n_layers_attention=La, q=_ptr(q).value, k_new=k_new.data_ptr(), v_new=v_new.data_ptr(),
                           hidden=hidden.data_ptr(), attn_out=_ptr(attn_out).value, step_scores_out=scores.data_ptr(),
                           scorer=C.pointer(weights.struct), threshold=threshold, keep_frac=keep_frac, max_evictions=max_evictions, check_every=check_every,
-                          score_history=_ptr(score_history).value)
+                          score_history=_ptr(score_history).value, use_graphs=int(bool(use_graphs)))
         r = step_run_result()
         _check("algorithm1_run", lib().algorithm1_run(self.handle, C.byref(a), C.byref(r), _stream(stream)))
         return {k: getattr(r, k) for k, _ in step_run_result._fields_}

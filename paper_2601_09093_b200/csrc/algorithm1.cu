@@ -20,6 +20,8 @@
 
 #include <string.h>
 
+#include <vector>
+
 using namespace stepk;
 
 namespace {
@@ -208,12 +210,21 @@ int algorithm1_run(step_pool* pool, const step_run_args* a, step_run_result* res
   const size_t q_slot = (size_t)La * n * g.Hq * g.d * eb;
   const size_t kv_slot = (size_t)n * g.L * g.Hkv * g.d * eb;
   const size_t h_slot = a->scorer ? (size_t)n * a->scorer->D * (a->scorer->dtype == STEP_BF16 ? 2 : 4) : 0;
+  // With use_graphs the launches of one iteration are recorded once per ring slot and replayed: what changes from
+  // one use of a slot to the next (the tokens, the row of the score history) goes through fixed staging rows.
+  bool graphs = a->use_graphs != 0 && s != nullptr && s != cudaStreamLegacy;
+  if (graphs) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) graphs = false;
+  }
+  std::vector<cudaGraphExec_t> execs(graphs ? a->ring : 0, nullptr);
+  auto drop_graphs = [&]() { for (cudaGraphExec_t e : execs) if (e) cudaGraphExecDestroy(e); };
   int done = 0, live = -1;
   for (int i = 0; i < a->max_iterations; ++i) {
     const int slot = i % a->ring;
     step_iteration it;
     it.n_traces = n;
-    it.token_ids = a->token_ids + (size_t)i * n;
+    it.token_ids = graphs ? pool->v.it_tokens : a->token_ids + (size_t)i * n;
     it.eos_token = a->eos_token;
     it.step_end_table = a->step_end_table; it.vocab = a->vocab;
     it.answers = a->answers;
@@ -229,16 +240,45 @@ int algorithm1_run(step_pool* pool, const step_run_args* a, step_run_result* res
     it.threshold = a->threshold; it.keep_frac = a->keep_frac;
     it.max_evictions = a->max_evictions;
     it.pruned_ids_out = nullptr; it.n_pruned_out = nullptr;
-    it.trace_scores_out = a->score_history ? a->score_history + (size_t)i * n : nullptr;
-    const int st = algorithm1_iteration(pool, &it, stream);
-    if (st != STEP_OK) return st;
+    float* hist_row = a->score_history ? a->score_history + (size_t)i * n : nullptr;
+    it.trace_scores_out = graphs ? (hist_row ? pool->v.it_scores : nullptr) : hist_row;
+    if (!graphs) {
+      const int st = algorithm1_iteration(pool, &it, stream);
+      if (st != STEP_OK) return st;
+    } else {
+      if (!execs[slot]) {
+        cudaGraph_t graph = nullptr;
+        if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { drop_graphs(); return STEP_ERR_CUDA; }
+        const int st = algorithm1_iteration(pool, &it, stream);
+        const cudaError_t e = cudaStreamEndCapture(s, &graph);          // always leaves capture mode
+        if (st != STEP_OK || e != cudaSuccess || !graph) {
+          if (graph) cudaGraphDestroy(graph);
+          drop_graphs();
+          cudaGetLastError();
+          return st != STEP_OK ? st : STEP_ERR_CUDA;
+        }
+        const cudaError_t e2 = cudaGraphInstantiate(&execs[slot], graph, 0);
+        cudaGraphDestroy(graph);
+        if (e2 != cudaSuccess) { execs[slot] = nullptr; drop_graphs(); return STEP_ERR_CUDA; }
+      }
+      cudaError_t e = cudaMemcpyAsync(pool->v.it_tokens, a->token_ids + (size_t)i * n, (size_t)n * sizeof(int32_t),
+                                      cudaMemcpyDeviceToDevice, s);
+      if (e == cudaSuccess) e = cudaGraphLaunch(execs[slot], s);
+      if (e == cudaSuccess && hist_row)
+        e = cudaMemcpyAsync(hist_row, pool->v.it_scores, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, s);
+      if (e != cudaSuccess) { drop_graphs(); return STEP_ERR_CUDA; }
+    }
     done = i + 1;
     if (done % a->check_every == 0 || done == a->max_iterations) {
       // the only host round trip of the loop: is anyone still live?
       const int st2 = kv_pool_stats(pool, nullptr, nullptr, nullptr, &live, stream);
-      if (st2 != STEP_OK) return st2;
+      if (st2 != STEP_OK) { drop_graphs(); return st2; }
       if (live == 0) break;
     }
+  }
+  if (graphs) {
+    if (cudaStreamSynchronize(s) != cudaSuccess) { drop_graphs(); return STEP_ERR_CUDA; }
+    drop_graphs();
   }
   int32_t* out = pool->v.it_pruned;                 // free between iterations: answer, count; weight as float bits
   const int st = weighted_vote(pool, out, reinterpret_cast<float*>(out + 1), out + 2, stream);

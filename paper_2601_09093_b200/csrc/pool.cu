@@ -65,6 +65,8 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.it_ids = take(T * 4);
   l.it_fin = take(T * 4);
   l.it_pruned = take(T * 4);
+  l.it_tokens = take(T * 4);
+  l.it_scores = take(T * 4);
   l.total = off;
   return l;
 }
@@ -340,6 +342,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.final_score = (float*)(m + lay.final_score); v.answer = (int32_t*)(m + lay.answer);
   v.finished = (uint8_t*)(m + lay.finished); v.it_ids = (int32_t*)(m + lay.it_ids);
   v.it_fin = (int32_t*)(m + lay.it_fin); v.it_pruned = (int32_t*)(m + lay.it_pruned);
+  v.it_tokens = (int32_t*)(m + lay.it_tokens); v.it_scores = (float*)(m + lay.it_scores);
   int st = kv_pool_reset(p, nullptr);
   if (st == STEP_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = STEP_ERR_CUDA;
   if (st != STEP_OK) { delete p; return st; }

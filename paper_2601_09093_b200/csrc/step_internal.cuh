@@ -42,7 +42,7 @@ struct MetaLayout {
   size_t score_idx, score_z, score_part;
   size_t attn_ml, attn_o, attn_cnt;
   size_t pre_ws_ml, pre_ws_o, pre_ml, pre_o;   // shared-prefix attention (zero-sized for pools the tensor-core kernel does not cover)
-  size_t final_score, answer, finished, it_ids, it_fin, it_pruned;
+  size_t final_score, answer, finished, it_ids, it_fin, it_pruned, it_tokens, it_scores;
   size_t total;
 };
 
@@ -56,6 +56,7 @@ struct DevViews {
   float* pre_ws_ml; float* pre_ws_o; float* pre_ml; float* pre_o;   // null when zero-sized
   float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
   int32_t* it_ids; int32_t* it_fin; int32_t* it_pruned;       // per-iteration lists of the Algorithm 1 driver
+  int32_t* it_tokens; float* it_scores;                       // staging rows of algorithm1_run's recorded iterations
 };
 
 }  // namespace stepk

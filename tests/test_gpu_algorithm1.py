@@ -184,3 +184,87 @@ def test_whole_run_in_one_call_against_the_oracle_replay():
         assert abs(fs[t] - s_) <= 1e-3 and int(vv["answer"][t].item()) == a_
     assert res["answer"] == ora.vote(final_scores=fs)
     assert pool.last_error()[1] == ora_pool.status == 0
+
+
+def test_iteration_can_be_captured_in_a_cuda_graph_and_replayed():
+    """algorithm1_iteration makes no host round trip, so one iteration per ring slot can be recorded as a CUDA graph and
+    replayed; the replayed run ends in exactly the state and outputs of the eagerly launched one."""
+    n, iters, ring, seed = 16, 48, 4, 31
+    pools = []
+    for _ in range(2):
+        cfg, vocab, eos, table, toks, answers, wx, wts, pool, _ = _driver_case(seed, n, iters, 40, False, p_eos=0.03)
+        pools.append((pool, wts))
+    gen = torch.Generator(device=DEV); gen.manual_seed(seed)
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    q, k, v, h = rnd(ring, 2, n, 8, 128), rnd(ring, n, 1, 2, 2, 128), rnd(ring, n, 1, 2, 2, 128), rnd(ring, n, cfg.scorer_D)
+    ans = torch.from_numpy(answers).to(DEV)
+    tok_slots = torch.zeros((ring, n), dtype=torch.int32, device=DEV)       # the graphs read the tokens from here
+    toks_dev = torch.from_numpy(toks).to(DEV)
+    outs = []
+    for pool, wts in pools:
+        outs.append(dict(att=torch.zeros((2, n, 8, 128), dtype=torch.float32, device=DEV),
+                         ys=torch.zeros(n, dtype=torch.float32, device=DEV),
+                         ts=torch.zeros(n, dtype=torch.float32, device=DEV)))
+
+    def one(pi, slot):
+        pool, wts = pools[pi]
+        o = outs[pi]
+        pool.algorithm1_iteration(tok_slots[slot], eos, table, ans, q[slot], k[slot], v[slot], h[slot], wts, 1.0, 0.5,
+                                  max_evictions=1, attn_out=o["att"], step_scores_out=o["ys"], trace_scores_out=o["ts"])
+
+    # first iterations eagerly on both pools (one-time set-up of the library happens outside any capture)
+    for i in range(ring):
+        tok_slots[i].copy_(toks_dev[i])
+        one(0, i); one(1, i)
+    torch.cuda.synchronize()
+    graphs = []
+    for slot in range(ring):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            one(1, slot)
+        graphs.append(g)
+    # capture recorded the launches without running them: pool 1 is still where pool 0 is
+    for i in range(ring, iters):
+        slot = i % ring
+        tok_slots[slot].copy_(toks_dev[i])
+        one(0, slot)
+        hist0 = {k_: t.clone() for k_, t in outs[0].items()}
+        graphs[slot].replay()
+        torch.cuda.synchronize()
+        for k_ in hist0:
+            assert torch.equal(torch.nan_to_num(hist0[k_], nan=-7.0), torch.nan_to_num(outs[1][k_], nan=-7.0)), (i, k_)
+    v0, v1 = pools[0][0].views(), pools[1][0].views()
+    for name in ("block_table", "seq_lens", "live", "refcount", "free_count", "trace_scores"):
+        assert torch.equal(v0[name], v1[name]), name
+    fc = int(v0["free_count"].item())
+    assert torch.equal(v0["free_list"][:fc], v1["free_list"][:fc])
+    s0, s1 = pools[0][0].stats(), pools[1][0].stats()
+    assert s0 == s1 and s0["live_traces"] < n
+    assert pools[0][0].last_error() == (0, 0) and pools[1][0].last_error() == (0, 0)
+
+
+def test_whole_run_with_recorded_iterations_equals_the_directly_launched_run():
+    """algorithm1_run(use_graphs) replays one CUDA graph per ring slot; results, history and pool state are those of
+    the run that launches every kernel itself."""
+    n, iters, ring, seed = 24, 120, 5, 33
+    runs = []
+    for use_graphs in (False, True):
+        cfg, vocab, eos, table, toks, answers, wx, wts, pool, _ = _driver_case(seed, n, iters, 28, False, p_eos=0.02)
+        gen = torch.Generator(device=DEV); gen.manual_seed(seed)
+        rnd = lambda *shape: torch.randn(shape, generator=gen, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+        q, k, v, h = rnd(ring, 2, n, 8, 128), rnd(ring, n, 1, 2, 2, 128), rnd(ring, n, 1, 2, 2, 128), rnd(ring, n, cfg.scorer_D)
+        hist = torch.full((iters, n), float("nan"), dtype=torch.float32, device=DEV)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            res = pool.algorithm1_run(torch.from_numpy(toks).to(DEV), eos, table, torch.from_numpy(answers).to(DEV), q, k, v, h,
+                                      wts, 1.0, 0.5, max_evictions=1, check_every=8, score_history=hist, use_graphs=use_graphs)
+        torch.cuda.synchronize()
+        runs.append((res, hist, pool))
+    (r0, h0, p0), (r1, h1, p1) = runs
+    assert r0 == r1 and r0["n_evicted"] >= 2 and r0["n_finished"] >= 2
+    assert torch.equal(torch.nan_to_num(h0, nan=-7.0), torch.nan_to_num(h1, nan=-7.0))
+    v0, v1 = p0.views(), p1.views()
+    for name in ("block_table", "seq_lens", "live", "refcount", "free_count", "trace_scores"):
+        assert torch.equal(v0[name], v1[name]), name
+    assert p0.last_error() == (0, 0) and p1.last_error() == (0, 0)
