@@ -564,6 +564,23 @@ def scorer_measurements(cfg, dev, rows=65536, reps=20, all_rows_density=1.0):
     code, mask_bits = pool.last_error()
     res["device_error_mask"] = mask_bits
     pool.close()
+    # one optimisation step of the scorer at the paper's batch size (128 labelled step-end hidden states)
+    Bt = 128
+    tr = B.ScorerTrainer(wts.W1.float(), wts.b1.float(), wts.w2.float(), wts.b2, batch=Bt, pos_weight=2.0)
+    labels = (torch.arange(Bt, device=dev) % 3 == 0).float()
+    for _ in range(3):
+        tr.step(hid[:Bt], labels)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for i in range(reps):
+        tr.step(hid[:Bt], labels)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(reps)]))
+    n_par = cfg.scorer_m * cfg.scorer_D + 2 * cfg.scorer_m + 1
+    res["train_step"] = {"batch": Bt, "us_per_step": ms * 1e3, "loss": float(tr.loss.item()),
+                         "gflops": 2 * 2.0 * Bt * cfg.scorer_m * cfg.scorer_D / (ms * 1e-3) / 1e9,
+                         "adam_bytes": n_par * 28, "launches": 5}
     return res
 
 

@@ -9,7 +9,8 @@
 //
 // Parameters, moments and gradients are fp32.  The batch is small (the paper trains with 128 rows), so the two
 // products (B x m x D each) are plain fp32 tiled GEMMs on CUDA cores: forward split over K across CTAs with the
-// partial sums added in a fixed order, backward as a rank-B update with one CTA per 64 x 64 tile of dW1.
+// partial sums added in a fixed order, backward as a rank-B update with one CTA per 64 x 64 tile of dW1.  Between
+// them a CTA per batch row makes the logit, loss term and dz, and a thread per hidden unit the small gradients.
 // Everything is deterministic (no floating-point atomics).
 #include "step_internal.cuh"
 
@@ -19,7 +20,8 @@ using namespace stepk;
 
 namespace {
 
-constexpr int kTile = 64, kKStep = 16, kSplitK = 8;
+constexpr int kTile = 64, kKStep = 16, kSplitK = 32;   // 32 K-slices: several CTAs per SM hide the load latency
+constexpr int kUnitRows = 16;                          // row slices of train_unit_kernel
 
 template <typename T> __device__ inline float ldf(const T* p);
 template <> __device__ inline float ldf<float>(const float* p) { return *p; }
@@ -36,13 +38,26 @@ train_fwd_kernel(const T* __restrict__ H, const float* __restrict__ W1, float* _
   const int k_lo = blockIdx.z * k_per, k_hi = min(D, k_lo + k_per);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   float acc[4][4] = {};
+  // the next tile's elements travel in registers while the current tile is multiplied
+  float ra[4], rb[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = threadIdx.x + q * 256, r = i / kKStep, k = k0 + i % kKStep;
+      ra[q] = (b0 + r < B && k < k_hi) ? ldf(H + (size_t)(b0 + r) * D + k) : 0.f;
+      rb[q] = (j0 + r < m && k < k_hi) ? W1[(size_t)(j0 + r) * D + k] : 0.f;
+    }
+  };
+  if (k_lo < k_hi) fetch(k_lo);
   for (int k0 = k_lo; k0 < k_hi; k0 += kKStep) {
-    for (int i = threadIdx.x; i < kTile * kKStep; i += 256) {
-      const int r = i / kKStep, kk = i % kKStep, k = k0 + kk;
-      sA[kk][r] = (b0 + r < B && k < k_hi) ? ldf(H + (size_t)(b0 + r) * D + k) : 0.f;
-      sB[kk][r] = (j0 + r < m && k < k_hi) ? W1[(size_t)(j0 + r) * D + k] : 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = threadIdx.x + q * 256;
+      sA[i % kKStep][i / kKStep] = ra[q];
+      sB[i % kKStep][i / kKStep] = rb[q];
     }
     __syncthreads();
+    if (k0 + kKStep < k_hi) fetch(k0 + kKStep);
 #pragma unroll
     for (int kk = 0; kk < kKStep; ++kk) {
       float av[4], bv[4];
@@ -65,62 +80,71 @@ train_fwd_kernel(const T* __restrict__ H, const float* __restrict__ W1, float* _
     }
 }
 
-// One CTA.  pre (slices added in order) -> z, loss, dz; then dw2, db2, db1 and dpre (written over part[0]).
-__global__ void __launch_bounds__(1024)
-train_loss_kernel(float* __restrict__ part, const float* __restrict__ labels, const float* __restrict__ b1,
-                  const float* __restrict__ w2, const float* __restrict__ b2, int B, int m, float pos_weight,
-                  float* __restrict__ dz, float* __restrict__ g_b1, float* __restrict__ g_w2, float* __restrict__ g_b2,
-                  float* __restrict__ loss_out) {
-  __shared__ float s_red[32];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  // pre-activations: fixed-order sum of the K slices, + b1; kept in part[0]
-  for (size_t i = threadIdx.x; i < (size_t)B * m; i += blockDim.x) {
+// One CTA per batch row: pre (slices added in order, + b1, kept in part[0]) -> z, the row's loss term and dz.
+__global__ void __launch_bounds__(256)
+train_row_kernel(float* __restrict__ part, const float* __restrict__ labels, const float* __restrict__ b1,
+                 const float* __restrict__ w2, const float* __restrict__ b2, int B, int m, float pos_weight,
+                 float* __restrict__ dz, float* __restrict__ loss_terms) {
+  __shared__ float s_red[8];
+  const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float z = 0.f;
+  for (int j = threadIdx.x; j < m; j += blockDim.x) {
+    const size_t i = (size_t)b * m + j;
     float p = 0.f;
     for (int s = 0; s < kSplitK; ++s) p += part[(size_t)s * B * m + i];
-    part[i] = p + b1[i % m];
+    p += b1[j];
+    part[i] = p;
+    z = fmaf(fmaxf(p, 0.f), w2[j], z);
   }
-  __syncthreads();
-  // a warp per row: z, its loss term and dz
-  float loss_acc = 0.f;
-  for (int b = warp; b < B; b += nwarps) {
-    float z = 0.f;
-    for (int j = lane; j < m; j += 32) z = fmaf(fmaxf(part[(size_t)b * m + j], 0.f), w2[j], z);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-    z += b2[0];
+  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+  if (lane == 0) s_red[warp] = z;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    z = b2[0];
+    for (int w = 0; w < 8; ++w) z += s_red[w];
     const float y = labels[b];
     // log sigmoid(z) = -softplus(-z), log(1 - sigmoid(z)) = -softplus(z), softplus(x) = max(x, 0) + log1p(exp(-|x|))
     const float sp_pos = fmaxf(z, 0.f) + log1pf(expf(-fabsf(z)));        // softplus(z)
     const float sp_neg = sp_pos - z;                                     // softplus(-z)
     const float sig = 1.f / (1.f + expf(-z));
-    if (lane == 0) {
-      loss_acc += pos_weight * y * sp_neg + (1.f - y) * sp_pos;
-      dz[b] = ((1.f - y) * sig - pos_weight * y * (1.f - sig)) / (float)B;
-    }
+    loss_terms[b] = pos_weight * y * sp_neg + (1.f - y) * sp_pos;
+    dz[b] = ((1.f - y) * sig - pos_weight * y * (1.f - sig)) / (float)B;
   }
-  if (lane == 0) s_red[warp] = loss_acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float l = 0.f;
-    for (int w = 0; w < nwarps; ++w) l += s_red[w];
-    *loss_out = l / (float)B;
-    float s = 0.f;
-    for (int b = 0; b < B; ++b) s += dz[b];
-    *g_b2 = s;
-  }
-  __syncthreads();
-  // per hidden unit: dw2, db1 (rows in order), and dpre in place
-  for (int j = threadIdx.x; j < m; j += blockDim.x) {
+}
+
+// dw2, db1 and dpre (in place) for 32 hidden units per CTA: thread (unit, slice) walks every kUnitRows-th row, the
+// slices are added in order through shared memory; thread 0 of CTA 0 adds up the loss and db2.
+__global__ void __launch_bounds__(32 * kUnitRows)
+train_unit_kernel(float* __restrict__ part, const float* __restrict__ w2, const float* __restrict__ dz,
+                  const float* __restrict__ loss_terms, int B, int m, float* __restrict__ g_b1, float* __restrict__ g_w2,
+                  float* __restrict__ g_b2, float* __restrict__ loss_out) {
+  __shared__ float s_gw[kUnitRows][32], s_gb[kUnitRows][32];
+  const int u = threadIdx.x & 31, r = threadIdx.x >> 5;
+  const int j = blockIdx.x * 32 + u;
+  float gw = 0.f, gb = 0.f;
+  if (j < m) {
     const float wj = w2[j];
-    float gw = 0.f, gb = 0.f;
-    for (int b = 0; b < B; ++b) {
+    for (int b = r; b < B; b += kUnitRows) {
       const float p = part[(size_t)b * m + j], d = dz[b];
       gw = fmaf(fmaxf(p, 0.f), d, gw);
       const float dp = p > 0.f ? d * wj : 0.f;
       gb += dp;
       part[(size_t)b * m + j] = dp;
     }
+  }
+  s_gw[r][u] = gw; s_gb[r][u] = gb;
+  __syncthreads();
+  if (r == 0 && j < m) {
+    gw = 0.f; gb = 0.f;
+    for (int q = 0; q < kUnitRows; ++q) { gw += s_gw[q][u]; gb += s_gb[q][u]; }
     g_w2[j] = gw; g_b1[j] = gb;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    float l = 0.f, sum = 0.f;
+    for (int b = 0; b < B; ++b) { l += loss_terms[b]; sum += dz[b]; }
+    *loss_out = l / (float)B;
+    *g_b2 = sum;
   }
 }
 
@@ -132,13 +156,25 @@ train_bwd_kernel(const float* __restrict__ dpre, const T* __restrict__ H, float*
   const int k0 = blockIdx.x * kTile, j0 = blockIdx.y * kTile;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   float acc[4][4] = {};
+  float ra[4], rb[4];
+  auto fetch = [&](int r0) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = threadIdx.x + q * 256, b = r0 + i / kTile, c = i % kTile;
+      ra[q] = (b < B && j0 + c < m) ? dpre[(size_t)b * m + j0 + c] : 0.f;
+      rb[q] = (b < B && k0 + c < D) ? ldf(H + (size_t)b * D + k0 + c) : 0.f;
+    }
+  };
+  fetch(0);
   for (int r0 = 0; r0 < B; r0 += kKStep) {
-    for (int i = threadIdx.x; i < kTile * kKStep; i += 256) {
-      const int rr = i / kTile, c = i % kTile, b = r0 + rr;
-      sA[rr][c] = (b < B && j0 + c < m) ? dpre[(size_t)b * m + j0 + c] : 0.f;
-      sB[rr][c] = (b < B && k0 + c < D) ? ldf(H + (size_t)b * D + k0 + c) : 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = threadIdx.x + q * 256;
+      sA[i / kTile][i % kTile] = ra[q];
+      sB[i / kTile][i % kTile] = rb[q];
     }
     __syncthreads();
+    if (r0 + kKStep < B) fetch(r0 + kKStep);
 #pragma unroll
     for (int rr = 0; rr < kKStep; ++rr) {
       float av[4], bv[4];
@@ -183,13 +219,14 @@ train_adam_kernel(float* __restrict__ W1, float* __restrict__ b1, float* __restr
   }
 }
 
-struct TrainLayout { size_t part, dz, g_W1, g_b1, g_w2, g_b2, total; };
+struct TrainLayout { size_t part, dz, loss_terms, g_W1, g_b1, g_w2, g_b2, total; };
 TrainLayout train_layout(int B, int D, int m) {
   TrainLayout l;
   size_t off = 0;
   auto take = [&](size_t floats) { size_t o = off; off += (floats * 4 + 255) / 256 * 256; return o; };
   l.part = take((size_t)kSplitK * B * m);
   l.dz = take(B);
+  l.loss_terms = take(B);
   l.g_W1 = take((size_t)m * D);
   l.g_b1 = take(m);
   l.g_w2 = take(m);
@@ -222,6 +259,7 @@ int scorer_train_step(const void* hidden, int hidden_dtype, const float* labels,
   char* ws = (char*)workspace;
   float* part = (float*)(ws + l.part);
   float* dz = (float*)(ws + l.dz);
+  float* loss_terms = (float*)(ws + l.loss_terms);
   float* g_W1 = (float*)(ws + l.g_W1);
   float* g_b1 = (float*)(ws + l.g_b1);
   float* g_w2 = (float*)(ws + l.g_w2);
@@ -232,7 +270,8 @@ int scorer_train_step(const void* hidden, int hidden_dtype, const float* labels,
     train_fwd_kernel<__nv_bfloat16><<<gf, 256, 0, s>>>((const __nv_bfloat16*)hidden, W1, part, B, D, m);
   else
     train_fwd_kernel<float><<<gf, 256, 0, s>>>((const float*)hidden, W1, part, B, D, m);
-  train_loss_kernel<<<1, 1024, 0, s>>>(part, labels, b1, w2, b2, B, m, h->pos_weight, dz, g_b1, g_w2, g_b2, loss_out);
+  train_row_kernel<<<B, 256, 0, s>>>(part, labels, b1, w2, b2, B, m, h->pos_weight, dz, loss_terms);
+  train_unit_kernel<<<(m + 31) / 32, 32 * kUnitRows, 0, s>>>(part, w2, dz, loss_terms, B, m, g_b1, g_w2, g_b2, loss_out);
   if (hidden_dtype == STEP_BF16)
     train_bwd_kernel<__nv_bfloat16><<<gb, 256, 0, s>>>(part, (const __nv_bfloat16*)hidden, g_W1, B, D, m);
   else
