@@ -43,7 +43,8 @@ def parse_args():
     ap.add_argument("--suffix-max", type=int, default=512, help="prefix workload: traces hold 1 .. this many tokens of their own")
     ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
     ap.add_argument("--scorer-density", type=float, default=1.0, help="fraction of those rows that end a step")
-    ap.add_argument("--scorer-shape", default="c1", choices=["c1", "c4"])
+    ap.add_argument("--scorer-shape", default="c1", choices=["c1", "c4", "d2560", "d5120"],
+                    help="scorer workload: D 4096 / m 512 (c1), D 5120 / m 1024 (c4), or the paper's other model widths with m 512")
     ap.add_argument("--traces", type=int, default=0, help="c3 only: sampling budget N (traces sharing the pool); 0 = 64")
     ap.add_argument("--threshold", type=float, default=0.0, help="c3 only: pool fraction at which the trigger fires; 0 = 0.95")
     ap.add_argument("--no-aux", action="store_true", help="skip the scorer / prune-cycle measurements after the timed steps")
@@ -697,6 +698,17 @@ def replay_cycles_on_oracle(cfg, nb, T, max_pages, append_log, snaps):
 
 
 # ---------------------------------------------------------------------------------------------
+def scorer_shape(name):
+    """The configuration whose scorer (D, m) the scorer workload uses; the paper's 4B and 14B-class models have
+    hidden sizes 2560 and 5120 with the same 512-unit scorer."""
+    from paper_2601_09093_b200 import workloads as W
+    if name == "d2560":
+        return W.scaled(W.C1, name="scorer-D2560-m512", scorer_D=2560)
+    if name == "d5120":
+        return W.scaled(W.C1, name="scorer-D5120-m512", scorer_D=5120)
+    return {"c1": W.C1, "c4": W.C4}[name]
+
+
 def run_scorer(args):
     """`--workload scorer`: score_steps alone on a large batch of step-end hidden states (every step of many
     finished traces scored at once).  The line's roofline is the tensor-core one of the first-layer GEMM."""
@@ -713,7 +725,7 @@ def run_scorer(args):
         dist.init_process_group("nccl", device_id=dev)
         dist.barrier()
     B.lib()
-    cfg = {"c1": W.C1, "c4": W.C4}[args.scorer_shape]
+    cfg = scorer_shape(args.scorer_shape)
     K = max(args.steps, 3)
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -881,7 +893,7 @@ def run_reference_scorer(args, K, Wm, sample=64):
     """The oracle's scorer on a bounded sample (64 step-end rows per step) of the batched scorer workload."""
     from oracle import scorer as OS
     from paper_2601_09093_b200 import workloads as W
-    cfg = {"c1": W.C1, "c4": W.C4}[args.scorer_shape]
+    cfg = scorer_shape(args.scorer_shape)
     (_, W1x), (_, b1x), (_, w2x), b2 = W.scorer_weights(cfg, bias_std=0.05)
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
     mask = np.ones(sample, dtype=np.uint8)
