@@ -124,3 +124,43 @@ def test_scorer_width_8192_runs_on_the_tensor_cores_only():
     with pytest.raises(B.StepError) as e:
         pool.score_steps(H.to_device(hb, "bf16"), torch.from_numpy(mask).cuda(), rt, wts)
     assert e.value.code == 1
+
+
+def test_shared_prefix_attention_at_the_trace_limit_and_beyond():
+    """2048 traces sharing one prompt page (G = 4: 512 bundles of 4) through decode_attention_shared_prefix; one trace
+    more is refused with nothing launched."""
+    n = 2048
+    cfg, tw = _many_short_traces(n, 37)
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (n, 8, 128), "bf16")
+    v = tw.gpu.views()
+    prefix = v["block_table"][5, :1].contiguous()
+    got = exact_f32(tw.gpu.decode_attention_shared_prefix(0, H.to_device(qb, "bf16"), v["block_table"], v["seq_lens"], prefix, 1))
+    want, short = OA.paged_decode_attention_shared_prefix(qx, tw.ora.k_pages[0], tw.ora.v_pages[0], tw.ora.block_table,
+                                                          tw.ora.seq_lens, tw.ora.block_table[5, :1])
+    mx, mean = attention_errors(got, want)
+    assert short == [] and mx <= 1e-2 and mean <= 1e-3
+    assert tw.status() == (0, 0)
+    cfg2, tw2 = _many_short_traces(2049, 38)
+    v2 = tw2.gpu.views()
+    q2 = torch.zeros((2049, 8, 128), dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(B.StepError):
+        tw2.gpu.decode_attention_shared_prefix(0, q2, v2["block_table"], v2["seq_lens"], v2["block_table"][0, :1].contiguous(), 1)
+    with pytest.raises(B.StepError):                              # more shared pages than a block-table row holds
+        tw.gpu.decode_attention_shared_prefix(0, H.to_device(qb, "bf16"), v["block_table"], v["seq_lens"], prefix, 5)
+
+
+def test_train_step_smallest_shapes():
+    """One hidden unit, one input dimension, three samples: the training kernels' tiles are almost entirely padding."""
+    from oracle import training as OT
+    H_ = np.array([[0.5], [-1.0], [2.0]]); y = np.array([1.0, 0.0, 1.0])
+    params = [np.array([[0.7]]), np.array([0.1]), np.array([-0.4]), np.array([0.05])]
+    opt = OT.Adam(params)
+    tr = B.ScorerTrainer(torch.tensor([[0.7]], device="cuda:0"), torch.tensor([0.1], device="cuda:0"),
+                         torch.tensor([-0.4], device="cuda:0"), 0.05, batch=3, pos_weight=0.5)
+    Hd = torch.tensor(H_, dtype=torch.float32, device="cuda:0"); yd = torch.tensor(y, dtype=torch.float32, device="cuda:0")
+    for _ in range(4):
+        lg = float(tr.step(Hd, yd).cpu()[0])
+        lo, params = OT.train_step(H_, y, params, opt, 0.5)
+        assert abs(lg - lo) <= 2e-5
+    for ref, got in zip(params, (tr.W1, tr.b1, tr.w2, tr.b2)):
+        np.testing.assert_allclose(got.cpu().numpy().reshape(ref.shape), ref, rtol=0, atol=5e-6)
