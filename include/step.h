@@ -207,7 +207,9 @@ int score_steps_tokens(step_pool* pool, const void* hidden, const int32_t* token
 int prune_if_saturated(step_pool* pool, const float* scores, float threshold, float keep_frac,
                        int32_t* pruned_ids_out, int32_t* n_pruned_out, void* stream);
 
-/* A trace that finished on its own gives its KV back (same reclaim as an eviction). */
+/* A trace that finished on its own gives its KV back (same reclaim as an eviction; the traces are reclaimed in the
+ * order listed, each one's pages in ascending order).  trace_ids: [n] device, distinct; invalid or dead ids are flagged
+ * (STEP_ERR_BAD_TRACE) and skipped. */
 int kv_pool_release_traces(step_pool* pool, const int32_t* trace_ids, int n, void* stream);
 
 /* ---- Algorithm 1 as a loop over device-resident state ----

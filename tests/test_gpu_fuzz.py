@@ -1,0 +1,91 @@
+"""Random sequences of pool operations on the CUDA pool and the oracle pool side by side: after every operation the
+free list, reference counts, block tables, lengths, live flags and status bits must be equal, bit for bit."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as OA
+from paper_2601_09093_b200 import harness as H
+from paper_2601_09093_b200 import workloads as W
+
+from gpu_common import Twin, exact_f32, attention_errors
+
+pytestmark = pytest.mark.gpu
+N_SEEDS = int(os.environ.get("STEP_FUZZ_SEEDS", "12"))
+
+
+def _dev(ids):
+    return torch.tensor(list(ids), dtype=torch.int32, device="cuda:0")
+
+
+@pytest.mark.parametrize("seed", range(N_SEEDS))
+def test_random_operation_sequences(seed):
+    g = np.random.default_rng(7000 + seed)
+    payload = seed % 3 == 0                                    # every third seed also carries K/V and checks attention
+    P = 16
+    cfg = W.scaled(W.C1, n_traces=24, num_layers=2, num_q_heads=8, num_kv_heads=2, prefix_len=0, seed=7000 + seed)
+    nb, max_pages, T = int(g.integers(40, 120)), int(g.integers(6, 14)), 24
+    tw = Twin(cfg, nb, max_pages, T, shuffle=bool(seed & 1), store_payload=payload)
+    o = tw.ora
+    n_ops = 60 if payload else 140
+    for step in range(n_ops):
+        live = [t for t in range(T) if o.live[t]]
+        op = g.choice(["fork", "append", "append", "append", "prune", "prune", "release", "finish"])
+        if op == "fork" or not live:
+            n = int(g.integers(1, 5))
+            plen = int(g.choice([0, 5, 16, 37, 48]))
+            full, rem = divmod(plen, P)
+            if o.next_trace + n > T or -(-plen // P) > max_pages or full + (n if rem else 0) > o.free_count or plen == 0 and payload:
+                continue                                       # forks that fail consume ids on one side only: not part of this test
+            ids, oids = tw.fork(n, plen)
+            assert ids == oids
+        elif op == "append":
+            k = int(g.integers(1, len(live) + 1))
+            ids = [int(x) for x in g.choice(live, size=k, replace=False)]
+            if g.random() < 0.15:
+                dead = [t for t in range(T) if not o.live[t]]
+                if dead:
+                    ids.insert(int(g.integers(0, len(ids) + 1)), int(g.choice(dead)))     # flagged and skipped on both sides
+            tw.append(ids, int(g.choice([1, 1, 2, 7, 16, 33])))
+        elif op == "prune":
+            scores = g.random(T).astype(np.float32)
+            if g.random() < 0.3:
+                scores[g.integers(0, T, size=3)] = scores[0]                                # ties
+            if g.random() < 0.2:
+                scores[g.integers(0, T)] = np.nan
+            thr = float(g.choice([0.3, 0.6, 0.9, 1.0]))
+            kf = float(g.choice([-1.0, 0.25, 0.5, 1.0]))
+            pid, pn = tw.gpu.prune_if_saturated(torch.from_numpy(scores).cuda(), thr, kf)
+            got = pid[:int(pn.item())].cpu().tolist()
+            assert got == o.prune_if_saturated(scores, thr, kf), (step, got)
+        elif op == "release":
+            ids = [int(x) for x in g.choice(live, size=int(g.integers(1, min(4, len(live)) + 1)), replace=False)]
+            tw.gpu.release_traces(_dev(ids))
+            for t in ids:                                      # reclaimed in the order listed
+                o.release_trace(t)
+        else:
+            ids = [int(x) for x in g.choice(live, size=int(g.integers(1, min(3, len(live)) + 1)), replace=False)]
+            tw.gpu.finish_traces(_dev(ids), _dev(g.integers(0, 4, size=len(ids))))
+            for t in ids:                                      # reclaimed in the order listed
+                o.release_trace(t)
+        try:
+            tw.assert_meta_equal()
+        except AssertionError as e:
+            v = tw.gpu.views()
+            fc = int(v["free_count"].item())
+            raise AssertionError("step %d op %s ids %s: %s\n gpu free %s\n ora free %s" % (
+                step, op, locals().get("ids"), e, v["free_list"][:fc].cpu().tolist(), o.free_list))
+        mask, omask = tw.status()
+        assert mask == omask, (step, op, mask, omask)
+    if payload:
+        n = o.next_trace
+        if n:
+            qb, qx = W.normal(cfg.seed, W.TID_Q, (n, 8, 128), "bf16")
+            v = tw.gpu.views()
+            for layer in (0, 1):
+                got = exact_f32(tw.gpu.decode_attention(layer, H.to_device(qb, "bf16"), v["block_table"][:n], v["seq_lens"][:n]))
+                want = OA.paged_decode_attention(qx, o.k_pages[layer], o.v_pages[layer], o.block_table[:n], o.seq_lens[:n])
+                mx, mean = attention_errors(got, want)
+                assert mx <= 1e-2 and mean <= 1e-3
