@@ -89,3 +89,66 @@ def test_random_operation_sequences(seed):
                 want = OA.paged_decode_attention(qx, o.k_pages[layer], o.v_pages[layer], o.block_table[:n], o.seq_lens[:n])
                 mx, mean = attention_errors(got, want)
                 assert mx <= 1e-2 and mean <= 1e-3
+
+
+@pytest.mark.parametrize("seed", range(N_SEEDS))
+def test_random_scorer_launches(seed):
+    """Random scorer widths, row counts, step-end densities and row-to-trace maps through score_steps (whichever
+    first-layer kernel the library picks) against the oracle."""
+    from test_gpu_parity import _scorer_case
+    g = np.random.default_rng(9000 + seed)
+    D = int(g.choice([64, 128, 320, 1000, 1024, 2560]))
+    m = int(g.choice([8, 64, 96, 128, 192, 512]))
+    T = int(g.integers(1, 70))
+    M = int(g.choice([1, 7, 128, 129, 255, 300, 1000, 2500]))
+    density = float(g.choice([0.0, 0.02, 0.3, 1.0]))
+    rt = g.integers(0, T, size=M).astype(np.int32) if g.random() < 0.7 or M > T else None
+    cfg = W.scaled(W.C1, n_traces=T, scorer_D=D, scorer_m=m, seed=9000 + seed)
+    chunk = int(g.choice([0, 0, 200])) if M > 200 else 0
+    _scorer_case(cfg, M, density, row_trace=rt, max_traces=T, max_score_rows=chunk or max(M, T),
+                 mode=int(g.choice([0, 0, 1, -1])))
+
+
+@pytest.mark.parametrize("seed", range(N_SEEDS))
+def test_random_attention_launches(seed):
+    """Random head groupings, trace counts, lengths (zeros and bare prompts included) and launch widths - so that the
+    cuts between the warps' partitions of the KV stream fall everywhere - through decode_attention, its shared-prefix
+    form and its allocation-free form, against the oracle."""
+    g = np.random.default_rng(11000 + seed)
+    hq, hkv = [(32, 8), (8, 8), (16, 2), (40, 8), (64, 8), (4, 1), (12, 4)][int(g.integers(0, 7))]
+    n = int(g.integers(1, 40))
+    prefix_len = int(g.choice([0, 9, 16, 50, 160]))
+    cfg = W.scaled(W.C1, n_traces=n, num_layers=1, num_q_heads=hq, num_kv_heads=hkv, prefix_len=prefix_len, seed=11000 + seed)
+    suffix = g.integers(0, int(g.choice([3, 40, 400])), size=n)
+    if prefix_len == 0:
+        suffix = np.maximum(suffix, 1)
+    pages = int(sum(-(-(prefix_len + int(x)) // 16) for x in suffix)) + 8
+    tw = Twin(cfg, pages, -(-(prefix_len + int(suffix.max())) // 16) + 2, n, shuffle=bool(seed & 1))
+    ids, _ = tw.fork(n, prefix_len)
+    for sel, inc in H.ragged_append_plan(np.asarray(suffix)):
+        if inc > 0:
+            assert all(tw.append([ids[i] for i in sel], inc))
+    if n > 2 and g.random() < 0.5:                                     # a dead trace in the middle: length 0, table -1
+        dead = int(g.integers(0, n))
+        tw.gpu.release_traces(_dev([dead])); tw.ora.release_trace(dead)
+    tw.gpu.set_attention_config(grid_ctas=int(g.integers(1, 149)))
+    o, v = tw.ora, tw.gpu.views()
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (n, hq, 128), "bf16")
+    qd = H.to_device(qb, "bf16")
+    want = OA.paged_decode_attention(qx, o.k_pages[0], o.v_pages[0], o.block_table[:n], o.seq_lens[:n])
+    got = exact_f32(tw.gpu.decode_attention(0, qd, v["block_table"][:n], v["seq_lens"][:n]))
+    mx, mean = attention_errors(got, want)
+    assert mx <= 1e-2 and mean <= 1e-3, ("plain", mx, mean)
+    if hq // hkv <= 8:
+        out = torch.empty((n, hq, 128), dtype=torch.float32, device="cuda:0")
+        tw.gpu.decode_attention_static(0, qd, v["block_table"][:n], v["seq_lens"][:n], out)
+        mx, mean = attention_errors(exact_f32(out), want)
+        assert mx <= 1e-2 and mean <= 1e-3, ("static", mx, mean)
+    pp = prefix_len // 16
+    live = [t for t in range(n) if o.live[t]]
+    if pp and live:
+        prefix = v["block_table"][live[0], :pp].contiguous()
+        got = exact_f32(tw.gpu.decode_attention_shared_prefix(0, qd, v["block_table"][:n], v["seq_lens"][:n], prefix, pp))
+        mx, mean = attention_errors(got, want)
+        assert mx <= 1e-2 and mean <= 1e-3, ("shared", mx, mean)
+    assert tw.status() == (0, 0)
