@@ -1,4 +1,4 @@
-"""CPU oracle for the STEP hot path (decode attention, step scorer, prune).
+"""CPU oracle for the STEP hot path (decode attention, step scorer, prune) and what was built around it.
 
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, obviously-correct
 restatement of what the method computes, written from the paper's equations
@@ -15,7 +15,11 @@ scorer.py     step scorer y = sigmoid(W2 ReLU(W1 h + b1) + b2) (Sec. 3.1,
               (Sec. 3.3, running-average equation).
 kv_pool.py    paged KV pool bookkeeping: InitTraces prefix fork, append,
               the memory trigger and the evict-lowest-score rule of
-              Algorithm 1 / Sec. 3.2, block reclaim.
+              Algorithm 1 / Sec. 3.2, block reclaim; the weighted vote.
+steps.py      step-end test of a sampled token's text (Sec. 3.1 footnote).
+algorithm1.py the loop of Algorithm 1 over the pieces above.
+training.py   weighted BCE-from-logits loss, its gradients and Adam for the
+              scorer (Sec. 3.1 "Training Objective"; appendix parameters).
 
 Every function is pinned by tests that do not re-use its own formula
 (brute force on unpaged data, closed forms, hand-worked examples,
