@@ -285,7 +285,8 @@ typedef struct {
                                          graph and replayed (one graph launch per iteration instead of a dozen kernel
                                          launches; worth it when an iteration is short).  Needs a stream that can be
                                          captured (not the default stream, not already capturing), else ignored.  The
-                                         graphs are private to the call and destroyed before it returns.              */
+                                         graphs are private to the call and destroyed before it returns (whatever memory
+                                         the CUDA runtime takes for them is the one exception to "allocates nothing"). */
 } step_run_args;
 
 typedef struct {
