@@ -66,3 +66,28 @@ def test_product_path_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src.replace("the oracle", "").replace("CPU oracle", ""), f
+
+
+def test_header_is_plain_c_and_struct_layouts_match_the_binding(tmp_path):
+    """include/step.h compiles as C99 on its own, and every struct the Python binding mirrors has the size and the
+    field offsets the C compiler gives it."""
+    import subprocess
+    from paper_2601_09093_b200 import binding as B
+    structs = ["kv_pool_config", "scorer_weights", "step_iteration", "step_run_args", "step_run_result", "scorer_train_hyper"]
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "step.h"', "int main(void) {"]
+    for s in structs:
+        lines.append('  printf("%s %%zu\\n", sizeof(%s));' % (s, s))
+        for name, _ in getattr(B, s)._fields_:
+            lines.append('  printf("%s.%s %%zu\\n", offsetof(%s, %s));' % (s, name, s, name))
+    lines += ["  return 0;", "}"]
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)],
+                   check=True)
+    out = dict(l.split() for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    for s in structs:
+        cls = getattr(B, s)
+        assert int(out[s]) == ctypes.sizeof(cls), s
+        for name, _ in cls._fields_:
+            assert int(out["%s.%s" % (s, name)]) == getattr(cls, name).offset, (s, name)
