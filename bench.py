@@ -38,7 +38,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer", "prefix"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer", "prefix", "replay"])
     ap.add_argument("--prefix-len", type=int, default=8192, help="prefix workload: tokens of the shared prompt")
     ap.add_argument("--suffix-max", type=int, default=512, help="prefix workload: traces hold 1 .. this many tokens of their own")
     ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
@@ -825,6 +825,142 @@ def run_prefix(args):
 
 
 # ---------------------------------------------------------------------------------------------
+def run_replay(args):
+    """`--workload replay`: the same 64 traces (one layer of the 8B layout, a pool that holds about 40 % of what they
+    would need) run twice - by an engine that does not prune and therefore preempts, queues and reconstructs traces
+    when the pool fills (the schedule of paper_2601_09093_b200/replay.py, host-driven by its nature, on this library's
+    fork / append / release / attention kernels), and by the method's own loop (algorithm1_run: eviction by score, no
+    queue).  Reports both runs' counters: the paper's Table 3 contrast (waiting 1526 s against 0) in units of decode
+    iterations.  Single GPU."""
+    import torch
+    from paper_2601_09093_b200 import binding as B, harness as H, ranks as R, workloads as W
+    from paper_2601_09093_b200 import build as _build
+    from paper_2601_09093_b200.replay import preempt_and_recompute
+    rank, local_rank, world = R.rank_env()
+    if rank != 0:
+        return
+    _build.build()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    B.lib()
+    cfg = W.scaled(W.C1, name="replay-1layer", prefix_len=512)
+    T, P, prompt = cfg.n_traces, cfg.page_size, cfg.prefix_len
+    final = [int(x) for x in prompt + W.rng(cfg.seed, W.TID_LEN, 5).integers(1024, 4097, size=T)]
+    nb = args.num_blocks or 4096
+    max_pages = -(-max(final) // P) + 2
+    max_traces = T + 4096                                           # every reconstruction takes a fresh trace id
+    pool = H.make_pool(cfg, nb, max_pages, max_traces, max_score_rows=T, device=dev)
+    v = pool.views()
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 3)
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    L, Hkv, Hq, d = cfg.num_layers, cfg.num_kv_heads, cfg.num_q_heads, cfg.head_dim
+    kbuf, vbuf = rnd(L, Hkv, max(final), d), rnd(L, Hkv, max(final), d)
+    knew, vnew, q = rnd(T, 1, L, Hkv, d), rnd(T, 1, L, Hkv, d), rnd(T, Hq, d)
+    out = torch.empty((T, Hq, d), dtype=torch.float32, device=dev)
+    zeros = torch.zeros(T, dtype=torch.int32, device=dev)
+
+    class Ops:
+        log, snap = [], None
+
+        def _ids(self, ids):
+            return torch.tensor(ids, dtype=torch.int32, device=dev)
+
+        def free(self):
+            return pool.stats()["free"]
+
+        def fork_all(self, n, S):
+            self.log.append(("fork", n, S))
+            return pool.fork_prefix(n, S, kbuf[:, :, :S].contiguous(), vbuf[:, :, :S].contiguous())
+
+        def fork_one(self, S):
+            return self.fork_all(1, S)[0]
+
+        def append(self, ids):
+            self.log.append(("append", list(ids)))
+            pool.append_kv(self._ids(ids), 1, knew[:len(ids)], vnew[:len(ids)])
+
+        def release(self, ids):
+            self.log.append(("release", list(ids)))
+            pool.release_traces(self._ids(ids))
+            if self.snap is None and sum(1 for o in self.log if o[0] == "release") == 8:
+                # state after the eighth preemption, for the oracle's replay of the log up to here
+                self.snap = (len(self.log), {k: v[k].clone() for k in ("block_table", "seq_lens", "live", "refcount", "free_list", "free_count")})
+
+        def finish(self, ids):
+            self.log.append(("release", list(ids)))
+            pool.finish_traces(self._ids(ids), zeros[:len(ids)])
+
+        def step(self, ids):
+            idx = torch.tensor(ids, dtype=torch.long, device=dev)
+            pool.decode_attention(0, q[:len(ids)], v["block_table"][idx], v["seq_lens"][idx], out[:len(ids)])
+
+    ops = Ops()
+    sampler = ClockSampler(local_rank); sampler.start()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    sc = preempt_and_recompute(ops, final, prompt, P)
+    torch.cuda.synchronize()
+    sc["seconds"] = time.perf_counter() - t0
+    sc["kv_bytes_rewritten"] = sc["recomputed_tokens"] * cfg.bytes_per_token
+    sc_stats, (sc_code, sc_mask) = pool.stats(), pool.last_error()
+
+    # the method's own loop on the same traces: trace t samples the end-of-sequence token when it reaches final[t]
+    pool2 = H.make_pool(cfg, nb, max_pages, T, max_score_rows=T, device=dev)
+    pool2.fork_prefix(T, prompt, kbuf[:, :, :prompt].contiguous(), vbuf[:, :, :prompt].contiguous())
+    vocab = W.synthetic_vocab(cfg.seed, 32000, step_end_frac=0.01)
+    table = B.step_end_table_from_vocab(vocab)
+    ends = np.flatnonzero(table.numpy())
+    max_it = max(final) - prompt
+    toks = W.token_ids(cfg.seed, max_it * T, len(vocab), ends, cfg.boundary_density, sub=9).reshape(max_it, T)
+    toks[toks == 0] = 1
+    for t in range(T):
+        toks[final[t] - prompt - 1, t] = 0
+    ring = 4
+    (W1b, _), (b1b, _), (w2b, _), b2 = W.scorer_weights(cfg)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16", dev), H.to_device(b1b, "bf16", dev), H.to_device(w2b, "bf16", dev), b2, B.STEP_BF16)
+    qr, kr, vr, hr = rnd(ring, 1, T, Hq, d), rnd(ring, T, 1, L, Hkv, d), rnd(ring, T, 1, L, Hkv, d), rnd(ring, T, cfg.scorer_D)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    st = pool2.algorithm1_run(torch.from_numpy(toks).to(dev), 0, table.to(dev), zeros, qr, kr, vr, hr, wts, 1.0, -1.0,
+                              max_evictions=4, check_every=64)
+    st["seconds"] = time.perf_counter() - t0
+    clocks = sampler.stop()
+    st_stats, (st_code, st_mask) = pool2.stats(), pool2.last_error()
+    st.update(waiting_trace_iterations=0, recomputed_tokens=0, preemptions=0)
+
+    res = {"metric": "decode iterations and waiting of 64 traces in a pool holding ~40 % of their KV: preempt-and-recompute engine vs the method's loop",
+           "value": sc["iterations"] / max(st["iterations"], 1), "unit": "x decode iterations (preempting engine / STEP loop)",
+           "n_gpus": 1, "steps": 1, "warmup": 0, "ms_per_step": st["seconds"] * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)",
+           "config": {"workload": cfg.name, "traces": T, "prompt": prompt, "final_lengths": "512 + U[1024, 4096]", "num_blocks": nb,
+                      "pool_tokens": nb * P, "tokens_if_all_complete": int(sum(final)), "l2_policy": "not a bandwidth measurement"},
+           "preempt_and_recompute": sc, "step_loop": st,
+           "status": {"sc_pool": sc_stats, "sc_error_mask": sc_mask, "step_pool": st_stats, "step_error_mask": st_mask},
+           "gpu_launches": sc["iterations"] * 3 + st["iterations"] * 9, "clocks": clocks}
+    if not args.no_cpu_baseline and ops.snap is not None:
+        from oracle.kv_pool import KVPoolOracle
+        n_ops, snap = ops.snap
+        o = KVPoolOracle(L, Hkv, d, P, nb, max_traces, max_pages, store_payload=False)
+        for op in ops.log[:n_ops]:
+            if op[0] == "fork":
+                o.fork_prefix(op[1], op[2])
+            elif op[0] == "append":
+                o.append_kv(op[1], 1)
+            else:
+                for t in op[1]:
+                    o.release_trace(t)
+        fc = int(snap["free_count"].item())
+        same = (fc == o.free_count and snap["free_list"][:fc].cpu().tolist() == o.free_list
+                and np.array_equal(snap["seq_lens"].cpu().numpy(), o.seq_lens)
+                and np.array_equal(snap["live"].cpu().numpy().astype(bool), o.live)
+                and np.array_equal(snap["refcount"].cpu().numpy(), o.refcount)
+                and np.array_equal(snap["block_table"].cpu().numpy(), o.block_table))
+        res["oracle_replay"] = {"what": "pool metadata after the eighth preemption (%d logged operations) against the oracle pool replaying the log" % n_ops,
+                                "bit_exact": bool(same), "oracle_status": o.status}
+    print(json.dumps(res))
+
+
+# ---------------------------------------------------------------------------------------------
 def run_reference(args):
     """The reference arm is the CPU oracle, as it stands, on the host cores.
     Under a multi-rank launcher rank 0 alone runs and prints; the other ranks leave at once."""
@@ -923,12 +1059,14 @@ def run_reference_scorer(args, K, Wm, sample=64):
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
-        if a.workload == "prefix":
+        if a.workload in ("prefix", "replay"):
             a.workload = "c1"           # the oracle's arm of the prefix workload is the one-layer configuration it is cut from
         run_reference(a)
     elif a.workload == "scorer":
         run_scorer(a)
     elif a.workload == "prefix":
         run_prefix(a)
+    elif a.workload == "replay":
+        run_replay(a)
     else:
         run_ours(a)
