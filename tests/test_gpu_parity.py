@@ -192,6 +192,23 @@ def test_attention_padding_slots_do_not_leak():
     _check_attention(tw, cfg, 2)
 
 
+@pytest.mark.parametrize("scale", [24.0, 1.0 / 64])
+def test_attention_with_peaked_and_flat_softmax(scale):
+    """Queries 24x larger make the softmax a near-argmax (logits of several hundred: only the max subtraction keeps
+    exp in range); queries 64x smaller make it a near-mean.  Both through the tensor-core and the scalar kernel."""
+    cfg = W.scaled(W.C1, n_traces=5, prefix_len=48, seed=515)
+    tw, ids = _build(cfg, [0, 7, 300, 1500, 64])
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (5, 32, 128), "bf16", std=scale)
+    want = _oracle_attention(tw, 0, qx, 5)
+    for fast in (1, -1):
+        tw.gpu.set_attention_config(fast_path=fast)
+        got = exact_f32(_gpu_attention(tw, 0, H.to_device(qb, "bf16"), 5))
+        assert np.isfinite(got).all()
+        mx, mean = attention_errors(got, want)
+        assert mx <= ATT_MAX and mean <= ATT_MEAN, (scale, fast, mx, mean)
+    assert tw.status() == (0, 0)
+
+
 def test_bad_block_table_is_flagged():
     cfg = W.scaled(W.C1, n_traces=1, prefix_len=32)
     tw, ids = _build(cfg, [40])
