@@ -404,3 +404,23 @@ def test_score_steps_tokens_equals_score_steps_on_the_oracle_mask(mode):
 def _exact_weights(cfg):
     (_, W1x), (_, b1x), (_, w2x), b2 = W.scorer_weights(cfg, bias_std=0.05)
     return W1x, b1x, w2x, b2
+
+
+@pytest.mark.parametrize("mode", [-1, 1])
+def test_scorer_saturating_logits(mode):
+    """Weights twenty times larger than usual drive the logit to tens or hundreds: the sigmoid must saturate to 0 / 1
+    without overflow or NaN, on the CUDA-core and on the tensor-core first layer."""
+    cfg = W.scaled(W.C1, n_traces=16, scorer_D=512, scorer_m=128, seed=616)
+    pool = H.make_pool(cfg, 8, 4, 16, max_score_rows=300)
+    pool.set_scorer_config(mode, 0)
+    (W1b, W1x), (b1b, b1x), (w2b, w2x), b2 = W.scorer_weights(cfg, std=1.0, bias_std=0.5)
+    wts = B.ScorerWeights(H.to_device(W1b, "bf16"), H.to_device(b1b, "bf16"), H.to_device(w2b, "bf16"), b2, B.STEP_BF16)
+    hb, hx = W.normal(cfg.seed, W.TID_HID, (300, 512), "bf16")
+    mask = np.ones(300, dtype=np.uint8)
+    rt = (np.arange(300) % 16).astype(np.int32)
+    got = pool.score_steps(H.to_device(hb, "bf16"), torch.from_numpy(mask).cuda(), torch.from_numpy(rt).cuda(), wts).cpu().numpy()
+    want = OS.score_steps(hx, mask, W1x, b1x, w2x, b2)
+    assert np.isfinite(got).all() and got.min() >= 0.0 and got.max() <= 1.0
+    assert (got == 0.0).any() or (got == 1.0).any() or (np.minimum(got, 1 - got).min() < 1e-6)      # it does saturate
+    assert np.abs(got - want).max() <= SCORE_TOL
+    assert pool.last_error() == (0, 0)
