@@ -98,6 +98,7 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
   const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
   __shared__ int s_warp[33];
   __shared__ int s_count, s_base, s_all;
+  dependents_may_launch();       // the first-layer kernel may set itself up on the other SMs meanwhile
   const float nan = __int_as_float(0x7fc00000);
   const int span = blockDim.x * kRowsPerThread;
   const int share = ((M + C - 1) / C + span - 1) / span * span;       // rows per CTA, whole passes
@@ -244,6 +245,7 @@ score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, in
   __shared__ int s_tr[kScoreFoldRows];
   __shared__ float2 s_run[kFinishThreads];
   __shared__ int s_last;
+  wait_for_primary();            // launched as a dependent of the first-layer kernel
   const int nb = v.counters[C_SCORE_NB], ns = v.counters[C_SCORE_SLICES];
   const int chunks = (nb + kScoreFoldRows - 1) / kScoreFoldRows;
   const int c = blockIdx.x;
@@ -421,8 +423,9 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
       if (st != STEP_OK) return st;
     }
     // row_trace == NULL means row i is trace i, counted from the start of the whole call
-    score_finish_kernel<<<(Mc + kScoreFoldRows - 1) / kScoreFoldRows, kFinishThreads, 0, s>>>(
-        pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off);
+    if (launch_dependent(score_finish_kernel, dim3((Mc + kScoreFoldRows - 1) / kScoreFoldRows), dim3(kFinishThreads), 0, s,
+                         pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off) != cudaSuccess)
+      return STEP_ERR_CUDA;
   }
   return launch_ok();
 }

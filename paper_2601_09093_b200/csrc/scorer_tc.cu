@@ -160,36 +160,6 @@ __device__ inline uint32_t umma_idesc_bf16(int n) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
-  // the launch decided on the device whether this kernel or the CUDA-core kernel scores its rows
-  const int N = a.counters[C_SCORE_TC];
-  if (N == 0) return;
-  const int nb = a.counters[C_SCORE_NB];
-  const int slices = a.m / N;
-  const int R = a.counters[C_SCORE_TILE];                       // rows per item: 256, or 128 for launches too small to
-  const int tiles = (nb + R - 1) / R;                           // fill the SMs with 256-row items
-  // operand ring: a stage holds R x 64 of the hidden rows and N x 64 of W1 (24 - 64 KiB), 3 to 8 stages
-  const int a_bytes = R / kHalfRows * kHalfBytes;
-  const int stage_bytes = a_bytes + N * kBK * 2;
-  const int n_stages = min(kMaxStages, kRingBytes / stage_bytes);
-  // Items are handed out round-robin, so a launch takes as long as the CTA with the most items.  With 256-row
-  // items the last round can be nearly empty; the rows that would make it up are cut into 128-row items instead,
-  // which spreads that last bit of work over twice as many CTAs.  (The ring keeps the 256-row stage layout.)
-  int n_big = tiles * slices, n_big_tiles = tiles, n_small = 0;
-  if (R > kHalfRows && n_big > (int)gridDim.x && n_big % (int)gridDim.x != 0) {
-    n_big_tiles = n_big / (int)gridDim.x * (int)gridDim.x / slices;
-    n_big = n_big_tiles * slices;
-    n_small = (nb - n_big_tiles * R + kHalfRows - 1) / kHalfRows * slices;
-  }
-  const int items = n_big + n_small;
-  // item -> first listed row, rows (256 or 128), slice of hidden units
-  auto item_rows = [&](int item, int& row0, int& slice) -> int {
-    if (item < n_big) { const int t = item / slices; slice = item - t * slices; row0 = t * R; return R; }
-    const int j = item - n_big, t = j / slices;
-    slice = j - t * slices; row0 = n_big_tiles * R + t * kHalfRows;
-    return kHalfRows;
-  };
-  const int KC = a.D / kBK;
-
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles want 1024-byte alignment
@@ -227,7 +197,44 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
 
-  if (warp < kEpiWarps) {
+  // Everything above touched only this CTA's own shared and tensor memory and the weights; the row list and the
+  // launch's shape come from the compaction kernel, whose completion this kernel may have been scheduled ahead of.
+  dependents_may_launch();
+  wait_for_primary();
+  // the launch decided on the device whether this kernel or the CUDA-core kernel scores its rows
+  const int n_units = a.counters[C_SCORE_TC];
+  const bool active = n_units != 0;   // 0: the CUDA-core kernel scored this launch's rows (or there were none)
+  const int N = active ? n_units : kBoxRows;
+  const int nb = active ? a.counters[C_SCORE_NB] : 0;
+  const int slices = a.m / N;
+  const int R = active ? a.counters[C_SCORE_TILE] : kHalfRows;  // rows per item: 256, or 128 for launches too small to
+  const int tiles = (nb + R - 1) / R;                           // fill the SMs with 256-row items
+  // operand ring: a stage holds R x 64 of the hidden rows and N x 64 of W1 (24 - 64 KiB), 3 to 8 stages
+  const int a_bytes = R / kHalfRows * kHalfBytes;
+  const int stage_bytes = a_bytes + N * kBK * 2;
+  const int n_stages = min(kMaxStages, kRingBytes / stage_bytes);
+  // Items are handed out round-robin, so a launch takes as long as the CTA with the most items.  With 256-row
+  // items the last round can be nearly empty; the rows that would make it up are cut into 128-row items instead,
+  // which spreads that last bit of work over twice as many CTAs.  (The ring keeps the 256-row stage layout.)
+  int n_big = tiles * slices, n_big_tiles = tiles, n_small = 0;
+  if (R > kHalfRows && n_big > (int)gridDim.x && n_big % (int)gridDim.x != 0) {
+    n_big_tiles = n_big / (int)gridDim.x * (int)gridDim.x / slices;
+    n_big = n_big_tiles * slices;
+    n_small = (nb - n_big_tiles * R + kHalfRows - 1) / kHalfRows * slices;
+  }
+  const int items = n_big + n_small;
+  // item -> first listed row, rows (256 or 128), slice of hidden units
+  auto item_rows = [&](int item, int& row0, int& slice) -> int {
+    if (item < n_big) { const int t = item / slices; slice = item - t * slices; row0 = t * R; return R; }
+    const int j = item - n_big, t = j / slices;
+    slice = j - t * slices; row0 = n_big_tiles * R + t * kHalfRows;
+    return kHalfRows;
+  };
+  const int KC = a.D / kBK;
+
+  if (!active) {
+    // nothing to do but give the tensor memory back below
+  } else if (warp < kEpiWarps) {
     // ------------------------------------------------ read-out: second layer on the accumulators
     const int quarter = warp & 3, half = warp >> 2;
     int li = 0;
@@ -444,7 +451,8 @@ int score_tc_launch(step_pool* pool, const void* hidden, int Mc, const scorer_we
   int grid = pool->num_sms;
   if (max_items < grid) grid = (int)max_items;
   if (grid < 1) grid = 1;
-  score_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(map, a);
+  // a dependent launch: the CTAs set themselves up while the compaction kernel is still running
+  if (launch_dependent(score_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, map, a) != cudaSuccess) return STEP_ERR_CUDA;
   return launch_ok();
 }
 

@@ -121,6 +121,25 @@ __device__ inline void flag_error(int32_t* counters, int code) {
 
 inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? STEP_OK : STEP_ERR_CUDA; }
 
+// Programmatic dependent launch.  A kernel launched with launch_dependent() may be scheduled while the kernel before
+// it in the stream is still running (as soon as every CTA of that kernel has called dependents_may_launch() or has
+// exited); it must call wait_for_primary() before it touches anything the earlier kernel writes - the call returns
+// once that kernel has completed and its writes are visible.  Both calls do nothing in a kernel launched the plain way.
+__device__ inline void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ inline void wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... Params, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 // ---- pieces the Algorithm 1 driver (algorithm1.cu) chains together
 // append_kv with two extras: *n_dev (device, may be null) caps the number of listed traces on the device, and
 // src_by_id makes trace t read row t of k_new / v_new instead of row (position in the list).
