@@ -29,7 +29,7 @@ def _digest() -> str:
     files.append(os.path.join(os.path.dirname(HERE), "include", "step.h"))
     for f in files:
         with open(f, "rb") as fh:
-            h.update(f.encode() + b"\0" + fh.read())
+            h.update(os.path.basename(f).encode() + b"\0" + fh.read())    # names, not paths: the tree may be moved
     return h.hexdigest()
 
 

@@ -91,3 +91,17 @@ def test_header_is_plain_c_and_struct_layouts_match_the_binding(tmp_path):
         assert int(out[s]) == ctypes.sizeof(cls), s
         for name, _ in cls._fields_:
             assert int(out["%s.%s" % (s, name)]) == getattr(cls, name).offset, (s, name)
+
+
+def test_build_stamp_does_not_depend_on_where_the_tree_lives(tmp_path, monkeypatch):
+    """A copy of the sources elsewhere has the same digest, so a library built here is not rebuilt after the tree
+    has been moved or copied."""
+    import shutil
+    from paper_2601_09093_b200 import build
+    here = build._digest()
+    pkg = tmp_path / "elsewhere" / "paper_2601_09093_b200"
+    shutil.copytree(build.CSRC, pkg / "csrc")
+    shutil.copytree(os.path.join(ROOT, "include"), tmp_path / "elsewhere" / "include")
+    monkeypatch.setattr(build, "CSRC", str(pkg / "csrc"))
+    monkeypatch.setattr(build, "HERE", str(pkg))
+    assert build._digest() == here
