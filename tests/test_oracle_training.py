@@ -76,3 +76,23 @@ def test_training_separates_two_clusters():
     assert losses[-1] < 0.25 * losses[0]
     s = np.array([OS.step_score(h, params[0], params[1], params[2], float(params[3][0])) for h in H])
     assert s[y == 1].min() > s[y == 0].max()
+
+
+def test_first_adam_step_closed_form():
+    """With zero moments the first bias-corrected update is lr * g / (|g| + eps): every parameter moves by (almost)
+    exactly lr against the sign of its gradient, whatever the gradient's size; weight decay enters through g."""
+    p = [np.array([[0.5, -2.0]]), np.array([3.0])]
+    g = [np.array([[1e-3, -40.0]]), np.array([0.0])]
+    opt = OT.Adam(p, lr=1e-2, eps=1e-8, weight_decay=0.0)
+    q = opt.step(p, g)
+    np.testing.assert_allclose(q[0], [[0.5 - 1e-2 * 1e-3 / (1e-3 + 1e-8), -2.0 + 1e-2 * 40.0 / (40.0 + 1e-8)]], rtol=0, atol=1e-15)
+    assert q[1][0] == 3.0                                             # zero gradient, no decay: no move
+    opt = OT.Adam(p, lr=1e-2, eps=1e-8, weight_decay=0.1)
+    q = opt.step(p, g)
+    g_eff = 0.0 + 0.1 * 3.0                                           # decay times the parameter joins the gradient
+    assert abs(q[1][0] - (3.0 - 1e-2 * g_eff / (g_eff + 1e-8))) < 1e-15
+    # second step from the same gradient: m = (1 - b1^2) g / (1 - b1^2) = g, v likewise -> the same step again
+    r = OT.Adam([np.array([1.0])], lr=1e-3, weight_decay=0.0)
+    a = r.step([np.array([1.0])], [np.array([2.0])])
+    b = r.step(a, [np.array([2.0])])
+    assert abs((a[0][0] - 1.0) - (b[0][0] - a[0][0])) < 1e-12
