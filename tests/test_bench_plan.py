@@ -14,7 +14,7 @@ from paper_2601_09093_b200 import workloads as W  # noqa: E402
 
 @pytest.mark.parametrize("traces,threshold", [(0, 0.0), (16, 0.0), (32, 0.5), (32, 0.9)])
 def test_memory_saturated_plan_stays_below_the_trigger_during_the_timed_steps(traces, threshold):
-    steps_total = 3 + 10 + 13 + 4 + bench.ALG1_ITERATIONS + 3
+    steps_total = 3 + 10 + 13 + 4 + bench.ALG1_ITERATIONS + 3 + bench.ALG1_GRAPH_ITERATIONS + 2      # as run_ours counts them
     cfg, suffix, nb, max_pages, layers = bench.workload_plan("c3", 0, steps_total, None, traces, threshold)
     T, P = cfg.n_traces, cfg.page_size
     assert T == (traces or 64) and layers == 36 and nb == 65536
@@ -50,3 +50,8 @@ def test_ragged_append_plan_gives_every_trace_its_length():
         assert inc > 0 and list(sel) == sorted(sel)
         got[sel] += inc
     assert np.array_equal(got, lengths)
+
+
+def test_scorer_shapes_are_the_papers_model_widths():
+    got = {name: (bench.scorer_shape(name).scorer_D, bench.scorer_shape(name).scorer_m) for name in ("c1", "c4", "d2560", "d5120")}
+    assert got == {"c1": (4096, 512), "c4": (5120, 1024), "d2560": (2560, 512), "d5120": (5120, 512)}
