@@ -495,6 +495,14 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     torch.cuda.synchronize()
     torch.cuda.current_stream().wait_stream(side)
     ms_g = g0.elapsed_time(g1) / n_g
+    # the loop's attention launches follow one another as programmatic dependents; the outputs of its last iteration
+    # must be, bit for bit, what one plain decode_attention call per layer gives on the same (unchanged) state
+    vv = pool.views()
+    q_last = q[(n_g - 1) % len(sets)]
+    same = True
+    for l in range(phys_layers):
+        direct = pool.decode_attention(l, q_last[l], vv["block_table"], vv["seq_lens"])
+        same = same and bool(torch.equal(direct, attn_out[l]))
     # step-end detection alone
     n_tok = 1 << 22
     big = torch.from_numpy(W.token_ids(cfg.seed, n_tok, len(vocab), ends, cfg.boundary_density, sub=77)).to(dev)
@@ -516,6 +524,7 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
             "recorded_iterations": {"iterations": rg["iterations"], "ms_per_iteration": ms_g,
                                     "trace_decode_steps_per_s": T / (ms_g * 1e-3), "vs_direct_launches": ms / ms_g,
                                     "live_left": rg["live_left"]},
+            "attention_outputs_equal_plain_calls": same,
             "detect_step_ends": {"tokens": n_tok, "us_per_call": det_ms * 1e3, "tokens_per_s": n_tok / (det_ms * 1e-3),
                                  "gbs": n_tok * 5 / (det_ms * 1e-3) / 1e9},
             "device_error_mask": bits}

@@ -120,6 +120,16 @@ int decode_attention(step_pool* pool, int layer, const void* q,
                      const int32_t* block_table, const int32_t* seq_lens, int n,
                      void* out, void* stream);
 
+/* decode_attention of n_layers consecutive layers, layer0 .. layer0 + n_layers - 1, over the same block table and
+ * lengths: q [n_layers, n, num_q_heads, head_dim], out [n_layers, n, num_q_heads, head_dim] fp32.  The results are
+ * those of n_layers decode_attention calls, bit for bit.  For callers that hold the queries of several layers at once
+ * (NextToken is outside this library, so the loop of Algorithm 1 is given all layers' queries of an iteration: see
+ * algorithm1_iteration).  Every launch after the first is made a programmatic dependent of the one before it, so the
+ * SMs pass from layer to layer one by one and the KV stream does not drain at layer boundaries. */
+int decode_attention_layers(step_pool* pool, int layer0, int n_layers, const void* q,
+                            const int32_t* block_table, const int32_t* seq_lens, int n,
+                            void* out, void* stream);
+
 /* decode_attention for traces that share their first pages (the prompt pages kv_pool_fork_prefix allocates once for
  * all traces of a problem: Algorithm 1, InitTraces):
  *   out[i] = attention of q[i] over the prefix_pages * page_size positions stored in blocks prefix_blocks[0 ..

@@ -93,6 +93,7 @@ def lib():
     L.append_kv.argtypes = [vp, vp, i, i, vp, vp, vp]
     L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_static.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.decode_attention_layers.argtypes = [vp, i, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_shared_prefix.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
     L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
     L.score_steps_tokens.argtypes = [vp, vp, vp, vp, i, vp, i, C.POINTER(scorer_weights), vp, vp, vp]
@@ -224,6 +225,15 @@ class KVPool:
             out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
         _check("decode_attention", lib().decode_attention(self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens),
                                                           n, _ptr(out), _stream(stream)))
+        return out
+
+    def decode_attention_layers(self, layer0, q, block_table, seq_lens, out=None, stream=None):
+        """q: [n_layers, n, Hq, d] -> out [n_layers, n, Hq, d] fp32: layers layer0 .. layer0 + n_layers - 1."""
+        n_layers, n = q.shape[0], q.shape[1]
+        if out is None:
+            out = torch.empty((n_layers, n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
+        _check("decode_attention_layers", lib().decode_attention_layers(self.handle, layer0, n_layers, _ptr(q), _ptr(block_table),
+                                                                        _ptr(seq_lens), n, _ptr(out), _stream(stream)))
         return out
 
     def decode_attention_shared_prefix(self, layer, q, block_table, seq_lens, prefix_blocks, prefix_pages, out=None, stream=None):

@@ -172,12 +172,8 @@ int algorithm1_iteration(step_pool* pool, const step_iteration* it, void* stream
   st = append_kv_impl(pool, v.it_ids, n, 1, it->k_new, it->v_new, v.counters + C_IT_NLIVE, 1, s);
   if (st != STEP_OK) return st;
   // NextToken's attention, layer by layer (traces that are not live have length 0 and get zeros)
-  const size_t q_layer = (size_t)n * g.Hq * g.d * pool->elem_bytes, o_layer = (size_t)n * g.Hq * g.d * sizeof(float);
-  for (int l = 0; l < it->n_layers_attention; ++l) {
-    st = decode_attention(pool, l, (const char*)it->q + l * q_layer, v.block_table, v.seq_lens, n,
-                          (char*)it->attn_out + l * o_layer, stream);
-    if (st != STEP_OK) return st;
-  }
+  st = decode_attention_layers(pool, 0, it->n_layers_attention, it->q, v.block_table, v.seq_lens, n, it->attn_out, stream);
+  if (st != STEP_OK) return st;
   // `if x ends a step: y <- f(h); update score_t`
   FlagSource src{nullptr, it->token_ids, it->step_end_table, it->vocab, it->boundary_mask_out, v.live};
   st = score_steps_impl(pool, it->hidden, src, nullptr, n, it->scorer, it->step_scores_out, stream);

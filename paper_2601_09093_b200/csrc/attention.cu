@@ -271,26 +271,39 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   }
   __syncthreads();
 
-  // traces without any position get zeros (CTAs take the traces round-robin); in the suffix pass a trace that
-  // holds the prefix and nothing else gets the normalised prefix result
-  if constexpr (kMode != kPrefixPass) {
-    for (int t = blockIdx.x; t < n; t += gridDim.x)
-      if (s_cum[t + 1] == s_cum[t]) {
-        const bool prefix_only = kMode == kSuffixPass && a.seq_lens[t] >= a.pp * kP;
-        for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) {
-          float v = 0.f;
-          if (prefix_only) v = a.pre_o[(size_t)t * a.Hq * kD + k] / a.pre_ml[((size_t)t * a.Hq + k / kD) * 2 + 1];
-          a.out[(size_t)t * a.Hq * kD + k] = v;
+  // Nothing has been written yet, and nothing read so far is written by another launch of this kernel: when this
+  // launch was scheduled ahead of the completion of such a launch before it (a layer-by-layer sequence of calls made
+  // by the library itself), it may run up to its first write - of an output, a partial or a ticket - and must then
+  // wait for that launch, whose partials and tickets share the scratch.  A no-op for a launch made the plain way.
+  dependents_may_launch();
+  bool waited = false;
+  auto before_first_write = [&]() { if (!waited) { wait_for_primary(); waited = true; } };
+  // traces without any position get zeros (CTAs take the traces round-robin, every thread its share); in the suffix
+  // pass a trace that holds the prefix and nothing else gets the normalised prefix result
+  auto fill_empty_traces = [&]() {
+    if constexpr (kMode != kPrefixPass) {
+      for (int t = blockIdx.x; t < n; t += gridDim.x)
+        if (s_cum[t + 1] == s_cum[t]) {
+          const bool prefix_only = kMode == kSuffixPass && a.seq_lens[t] >= a.pp * kP;
+          for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) {
+            float v = 0.f;
+            if (prefix_only) v = a.pre_o[(size_t)t * a.Hq * kD + k] / a.pre_ml[((size_t)t * a.Hq + k / kD) * 2 + 1];
+            a.out[(size_t)t * a.Hq * kD + k] = v;
+          }
         }
-      }
-  }
+    }
+  };
 
   const long long total = (long long)Hkv * s_cum[n];
   const int n_part = gridDim.x * kWarps;
   const long long W = (total + n_part - 1) / n_part;
   const int part = blockIdx.x * kWarps + warp;
   const long long pos0 = (long long)part * W;
-  if (W == 0 || pos0 >= total) return;
+  if (W == 0 || pos0 >= total) {
+    before_first_write();
+    fill_empty_traces();
+    return;
+  }
   const int cnt = (int)((pos0 + W <= total ? pos0 + W : total) - pos0);
 
   unsigned char* my_pages = s_pages + (size_t)warp * kStages * kPageBytes;
@@ -480,6 +493,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
       }
       const bool complete = seg_first_page == 0 && cc.page + 1 == cc.np;
       const int R = kMode == kPrefixPass ? 16 : G;       // rows of a partial slot
+      before_first_write();
       if (complete && kMode == kPrefixPass) {
         // the bundle's whole prefix was read by this warp: (m, l, o) of every (trace, head) row, un-normalised
         const int ta = cc.t * a.tpb + g_row / G, tb = cc.t * a.tpb + (g_row + 8) / G;
@@ -618,6 +632,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     if (++stage == kStages) { stage = 0; parity ^= 1; }
   }
 
+  before_first_write();
+  fill_empty_traces();
   if (!alive) {
     // A wait ran out.  Copies already issued still target this CTA's shared memory, so give each
     // of them one more bounded wait before the warp leaves; nothing else is touched.
@@ -630,21 +646,28 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
 constexpr int kWarpsDefault = 8, kStagesDefault = 3;
 
+// dependent: the launch may be scheduled before the kernel ahead of it in the stream has completed (see the kernel's
+// note on its first write); only for a launch that directly follows another launch of this kernel on the same pool.
 template <int kWarps, int kStages, bool kRows16, int kMode>
-int launch_one(const AttnArgs& a, int grid, cudaStream_t s) {
+int launch_one(const AttnArgs& a, int grid, cudaStream_t s, bool dependent = false) {
   const size_t smem = (size_t)kWarps * kStages * kPageBytes + (size_t)kWarps * kStages * 8 + (size_t)(a.n + 1) * 4;
   auto kern = attn_mma_kernel<kWarps, kStages, kRows16, kMode>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
-  kern<<<grid, kWarps * 32, smem, s>>>(a);
+  if (dependent) {
+    if (launch_dependent(kern, dim3(grid), dim3(kWarps * 32), smem, s, a) != cudaSuccess) return STEP_ERR_CUDA;
+  } else {
+    kern<<<grid, kWarps * 32, smem, s>>>(a);
+  }
   return launch_ok();
 }
 
 template <int kWarps, int kStages, int kMode>
-int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s) {
+int launch_mma(const step_pool* pool, const AttnArgs& a, cudaStream_t s, bool dependent = false) {
   int grid = pool->attn_grid;
   if (grid * kWarps > kMaxPartitions) grid = kMaxPartitions / kWarps;
   if (grid < 1) grid = 1;
-  return a.G > 8 ? launch_one<kWarps, kStages, true, kMode>(a, grid, s) : launch_one<kWarps, kStages, false, kMode>(a, grid, s);
+  return a.G > 8 ? launch_one<kWarps, kStages, true, kMode>(a, grid, s, dependent)
+                 : launch_one<kWarps, kStages, false, kMode>(a, grid, s, dependent);
 }
 
 void fill_args(AttnArgs& a, const step_pool* pool, const Geo& g, int layer, const void* q, const int32_t* block_table,
@@ -664,8 +687,37 @@ bool mma_shape(const step_pool* pool, const Geo& g, int n) {
 
 }  // namespace
 
+static int decode_attention_launch(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                   const int32_t* seq_lens, int n, void* out, void* stream, bool dependent);
+
 extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const int32_t* block_table,
                                 const int32_t* seq_lens, int n, void* out, void* stream) {
+  return decode_attention_launch(pool, layer, q, block_table, seq_lens, n, out, stream, false);
+}
+
+// decode_attention of several consecutive layers whose queries the caller has at hand.  The first layer's launch is an
+// ordinary one; every later launch directly follows the launch of the layer before it, reads nothing that one writes,
+// and is therefore made its programmatic dependent: an SM that has finished its share of layer l starts on layer l + 1
+// at once instead of idling until the whole of layer l is done, and the stream of KV reads never drains at a layer
+// boundary (the kernel holds its first write back until the launch before it has completed).
+extern "C" int decode_attention_layers(step_pool* pool, int layer0, int n_layers, const void* q,
+                                       const int32_t* block_table, const int32_t* seq_lens, int n, void* out,
+                                       void* stream) {
+  if (!pool || n < 0 || n_layers < 0 || layer0 < 0) return STEP_ERR_INVALID_ARG;
+  if (n == 0 || n_layers == 0) return STEP_OK;
+  if (layer0 + n_layers > pool->cfg.num_layers) return STEP_ERR_INVALID_ARG;
+  const size_t q_layer = (size_t)n * pool->cfg.num_q_heads * pool->cfg.head_dim * pool->elem_bytes;
+  const size_t o_layer = (size_t)n * pool->cfg.num_q_heads * pool->cfg.head_dim * sizeof(float);
+  for (int l = 0; l < n_layers; ++l) {
+    const int st = decode_attention_launch(pool, layer0 + l, q ? (const char*)q + l * q_layer : nullptr, block_table, seq_lens, n,
+                                           out ? (char*)out + l * o_layer : nullptr, stream, l > 0);
+    if (st != STEP_OK) return st;
+  }
+  return STEP_OK;
+}
+
+static int decode_attention_launch(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                   const int32_t* seq_lens, int n, void* out, void* stream, bool dependent) {
   if (!pool || n < 0) return STEP_ERR_INVALID_ARG;
   if (n == 0) return STEP_OK;
   if (!q || !block_table || !seq_lens || !out) return STEP_ERR_INVALID_ARG;
@@ -675,7 +727,7 @@ extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const
   if (pool->fast_path > 0 && mma_shape(pool, g, n)) {
     AttnArgs a;
     fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
-    return launch_mma<kWarpsDefault, kStagesDefault, kPlain>(pool, a, s);
+    return launch_mma<kWarpsDefault, kStagesDefault, kPlain>(pool, a, s, dependent);
   }
   if (n > 65535) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)(g.d + kScalarWarps * g.d) * sizeof(float);

@@ -424,3 +424,31 @@ def test_scorer_saturating_logits(mode):
     assert (got == 0.0).any() or (got == 1.0).any() or (np.minimum(got, 1 - got).min() < 1e-6)      # it does saturate
     assert np.abs(got - want).max() <= SCORE_TOL
     assert pool.last_error() == (0, 0)
+
+
+@pytest.mark.parametrize("hq,hkv", [(32, 8), (32, 2)])
+def test_attention_layers_call_equals_layer_by_layer_calls(hq, hkv):
+    """decode_attention_layers (every launch after the first a programmatic dependent of the one before) gives, bit
+    for bit, what one decode_attention call per layer gives, and both agree with the oracle."""
+    cfg = W.scaled(W.C1, n_traces=9, num_layers=5, num_q_heads=hq, num_kv_heads=hkv, prefix_len=40, seed=717)
+    tw, ids = _build(cfg, [0, 300, 17, 1200, 64, 5, 900, 33, 2000])
+    tw.gpu.release_traces(torch.tensor([4], dtype=torch.int32, device="cuda")); tw.ora.release_trace(4)
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (5, 9, hq, 128), "bf16")
+    qd = H.to_device(qb, "bf16")
+    v = tw.gpu.views()
+    for grid in (148, 5):
+        tw.gpu.set_attention_config(grid_ctas=grid)
+        for layer0, nl in ((0, 5), (2, 3), (4, 1)):
+            got = tw.gpu.decode_attention_layers(layer0, qd[:nl], v["block_table"][:9], v["seq_lens"][:9])
+            for l in range(nl):
+                one = tw.gpu.decode_attention(layer0 + l, qd[l], v["block_table"][:9], v["seq_lens"][:9])
+                assert torch.equal(got[l], one), (grid, layer0, l)
+                want = _oracle_attention(tw, layer0 + l, qx[l], 9)
+                mx, mean = attention_errors(exact_f32(got[l]), want)
+                assert mx <= ATT_MAX and mean <= ATT_MEAN
+    # many short launches in a row: every launch's partials and tickets share one scratch area
+    big = torch.stack([tw.gpu.decode_attention_layers(0, qd, v["block_table"][:9], v["seq_lens"][:9]).clone() for _ in range(20)])
+    assert all(torch.equal(big[0], b) for b in big[1:])
+    assert tw.status() == (0, 0)
+    with pytest.raises(B.StepError):
+        tw.gpu.decode_attention_layers(3, qd[:3], v["block_table"][:9], v["seq_lens"][:9])     # layers 3, 4, 5: one too many
