@@ -219,16 +219,20 @@ def run_ours(args):
 
     ids_host = list(ids)
 
+    # the logical layers as runs of consecutive resident layers (one run unless fewer layers are resident than the model has)
+    layer_runs = [(l0, min(phys_layers, L - l0)) for l0 in range(0, L, phys_layers)]
+
     def hot_path(s, time_attn=False, out=out, step_scores=step_scores):
         pool.append_kv(ids_dev, 1, s["k"], s["v"])
         append_log.append((ids_host, 1))
-        for l in range(L):
+        for l0, nl in layer_runs:
             if time_attn:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-            pool.decode_attention(l % phys_layers, s["q"][l], v["block_table"], v["seq_lens"], out[l])
+            # all layers of the run in one call: each launch a programmatic dependent of the one before it
+            pool.decode_attention_layers(0, s["q"][l0:l0 + nl], v["block_table"], v["seq_lens"], out[l0:l0 + nl])
             if time_attn:
-                e1.record(stream); attn_events.append((e0, e1))
+                e1.record(stream); attn_events.append((e0, e1, nl))
         pool.score_steps(s["h"], s["m"], None, wts, step_scores)
         pool.prune_if_saturated(None, cfg.threshold, cfg.keep_frac)
 
@@ -308,7 +312,21 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms_total = ev0.elapsed_time(ev1)
-    attn_ms = [a.elapsed_time(b) for a, b in attn_events]
+    attn_run_ms = [a.elapsed_time(b) for a, b, _ in attn_events]
+    attn_ms = [t / nl for t, (_, _, nl) in zip(attn_run_ms, attn_events)]     # per launch, within its run of layers
+    attn_launches = sum(nl for _, _, nl in attn_events)
+    # the same kernel launched alone (plain decode_attention calls, one event pair each), for comparison
+    iso = []
+    for i in range(2 + 12):                                              # two untimed launches first
+        l = i % phys_layers
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        pool.decode_attention(l, sets[0]["q"][l], v["block_table"], v["seq_lens"], out[l])
+        e1.record(stream)
+        if i >= 2:
+            iso.append((e0, e1))
+    torch.cuda.synchronize()
+    iso_ms = float(np.mean([a.elapsed_time(b) for a, b in iso]))
     err_code, err_mask = pool.last_error()
     n_live = pool.stats()["live_traces"]
     seq_now = v["seq_lens"][:T].cpu().numpy().astype(np.int64)
@@ -344,7 +362,7 @@ def run_ours(args):
     kv_bytes = H.unique_kv_bytes(cfg, cfg.prefix_len, mid_suffix)
     pages = int(np.sum(-(-(mid_suffix + cfg.prefix_len) // cfg.page_size)))
     algo_bytes = kv_bytes + T * cfg.num_q_heads * cfg.head_dim * (2 + 4) + pages * 4
-    attn_avg_ms = float(np.mean(attn_ms))
+    attn_avg_ms = float(np.sum(attn_run_ms)) / attn_launches
     achieved = algo_bytes / (attn_avg_ms * 1e-3) / 1e9
     value = R.whole_job_rate(T * K, world, ms_total * 1e-3)
     res = {
@@ -361,13 +379,20 @@ def run_ours(args):
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
                      "traffic": None if ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE is None else algo_bytes * ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE,
                      "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the one-layer 64-trace workload, scaled by algorithmic bytes",
-                     "kernel": "decode_attention (attn_mma_kernel, split partials merged in the same launch), one layer",
+                     "kernel": "decode_attention_layers (attn_mma_kernel, split partials merged in the same launch), per layer",
                      "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": attn_avg_ms,
-                     "min_launch_ms": float(np.min(attn_ms)), "launches_timed": len(attn_ms)},
+                     "min_launch_ms": float(np.min(attn_ms)), "launches_timed": attn_launches,
+                     "how_timed": "CUDA events around each decode_attention_layers call (all layers of a step: every launch after "
+                                  "the first is a programmatic dependent of the one before it, so launches overlap at layer "
+                                  "boundaries); avg_launch_ms = elapsed / launches.  The peak is a copy (reads and writes) of one "
+                                  "isolated launch; a read-only stream that never drains between launches can exceed it.",
+                     "isolated_launch": {"avg_launch_ms": iso_ms, "achieved": algo_bytes / (iso_ms * 1e-3) / 1e9,
+                                         "frac": algo_bytes / (iso_ms * 1e-3) / 1e9 / peak,
+                                         "what": "plain decode_attention calls timed one by one after the timed region"}},
         "kv_gbs": achieved,
         # the same launches counted the way a per-trace kernel would see them (the shared prompt once per trace)
         "kv_gbs_logical": float(np.sum(seq_now - K // 2)) * cfg.bytes_per_token_layer / (attn_avg_ms * 1e-3) / 1e9,
-        "attention_share_of_step": float(np.sum(attn_ms)) / ms_total,
+        "attention_share_of_step": float(np.sum(attn_run_ms)) / ms_total,
         "gpu_launches": K * (2 + L + 3 + 1), "clocks": clocks,
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
@@ -406,10 +431,13 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
     t_cpu, max_err, sum_err, cnt, done = 0.0, 0.0, 0.0, 0, 0
     wall0 = time.perf_counter()
+    # the outputs of every layer for the inputs in `s`, recomputed the way the timed steps launch them (runs of
+    # consecutive resident layers through decode_attention_layers) so that they are known to match these inputs
+    for l0 in range(0, L, phys_layers):
+        nl = min(phys_layers, L - l0)
+        pool.decode_attention_layers(0, s["q"][l0:l0 + nl], v["block_table"], v["seq_lens"], out[l0:l0 + nl])
+    torch.cuda.synchronize()
     for layer in layers[:L]:
-        # the output of this layer for the inputs in `s`, recomputed so that it is known to match them
-        pool.decode_attention(layer % phys_layers, s["q"][layer], v["block_table"], v["seq_lens"], out[layer])
-        torch.cuda.synchronize()
         got_all = out[layer].cpu().numpy().astype(np.float64)
         q_all = s["q"][layer].float().cpu().numpy().astype(np.float64)
         for t in range(T):
@@ -433,7 +461,7 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
     base = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "%d (trace, layer) attentions at full length, all heads (%.1f s of CPU), extrapolated to %d layers per step"
                       % (done, t_cpu, L)}
-    par = {"what": "decode_attention vs fp64 oracle on read-back KV: %d (trace, layer) pairs, all heads" % done,
+    par = {"what": "decode_attention_layers (the timed launch configuration) vs fp64 oracle on read-back KV: %d (trace, layer) pairs, all heads" % done,
            "max_abs_err": max_err, "mean_abs_err": sum_err / cnt, "tolerance": {"max": 1e-2, "mean": 1e-3},
            "ok": bool(max_err <= 1e-2 and sum_err / cnt <= 1e-3)}
     return base, par
