@@ -37,8 +37,14 @@ def _sampled_attention_parity(cfg, phys_layers, layer, sample_traces):
     H.fill_random_device(pool, cfg_pool, suffix, seed=cfg.seed, chunk_tokens=max(16, (1 << 28) // (T * cfg_pool.bytes_per_token)))
     v = pool.views()
     gen = torch.Generator(device="cuda"); gen.manual_seed(cfg.seed + 3)
-    q = torch.randn((T, cfg.num_q_heads, cfg.head_dim), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-    out = pool.decode_attention(layer, q, v["block_table"], v["seq_lens"]).cpu().numpy().astype(np.float64)
+    q_all = torch.randn((phys_layers, T, cfg.num_q_heads, cfg.head_dim), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    # all resident layers in one call, as the benchmark's step does: the checked layer's launch is then a programmatic
+    # dependent of the layer before it
+    out_all = pool.decode_attention_layers(0, q_all, v["block_table"], v["seq_lens"])
+    plain = pool.decode_attention(layer, q_all[layer], v["block_table"], v["seq_lens"])
+    assert torch.equal(out_all[layer], plain)
+    q = q_all[layer]
+    out = out_all[layer].cpu().numpy().astype(np.float64)
     assert pool.last_error() == (0, 0)
     seq = v["seq_lens"].cpu().numpy()
     assert np.array_equal(seq[:T], cfg.prefix_len + suffix)
@@ -61,13 +67,13 @@ def _sampled_attention_parity(cfg, phys_layers, layer, sample_traces):
 def test_c1_full_size_attention_sampled():
     """64 traces, 32/8 heads, 512 shared + U[4k,16k] tokens: shortest, longest and a few other traces."""
     s = W.suffix_lengths(W.C1)
-    _sampled_attention_parity(W.C1, 1, 0, sorted({int(np.argmin(s)), int(np.argmax(s)), 0, 31, 63}))
+    _sampled_attention_parity(W.C1, 2, 1, sorted({int(np.argmin(s)), int(np.argmax(s)), 0, 31, 63}))
 
 
 def test_c4_full_size_attention_sampled():
     """128 traces, 64/8 heads (G = 8), 1024 shared + log-uniform 1k-24k tokens."""
     s = W.suffix_lengths(W.C4)
-    _sampled_attention_parity(W.C4, 1, 0, sorted({int(np.argmin(s)), int(np.argmax(s)), 1, 64, 127}))
+    _sampled_attention_parity(W.C4, 2, 1, sorted({int(np.argmin(s)), int(np.argmax(s)), 1, 64, 127}))
 
 
 def test_c2_long_traces_shuffled_pages_sampled():
