@@ -59,7 +59,7 @@ def parse_args():
 # ncu capture on the one-layer 64-trace workload (2.6920 GB + 6.64 MB against 2.6628 GB algorithmic; the summary is
 # profiles/attn_mma_kernel_C1_ncu_full.md).  The kernel streams every page once, so traffic grows in proportion to
 # the algorithmic bytes and the larger workloads scale this figure.  Set to None when the kernel changes.
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (2.691363e9 + 6.766336e6) / 2.662836852e9
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = (2.692241e9 + 7.931648e6) / 2.662836852e9
 
 
 def measured_peaks(key="hbm_gbs", fallback=6650.0):
