@@ -125,7 +125,10 @@ int decode_attention(step_pool* pool, int layer, const void* q,
  * those of n_layers decode_attention calls, bit for bit.  For callers that hold the queries of several layers at once
  * (NextToken is outside this library, so the loop of Algorithm 1 is given all layers' queries of an iteration: see
  * algorithm1_iteration).  Every launch after the first is made a programmatic dependent of the one before it, so the
- * SMs pass from layer to layer one by one and the KV stream does not drain at layer boundaries. */
+ * SMs pass from layer to layer one by one and the KV stream does not drain at layer boundaries.  A later layer's launch
+ * may read its queries, the tables and the cache while an earlier layer is still writing its output: q, block_table
+ * and seq_lens must not overlap out.  Errors as decode_attention; layer0 + n_layers > num_layers is
+ * STEP_ERR_INVALID_ARG with nothing launched. */
 int decode_attention_layers(step_pool* pool, int layer0, int n_layers, const void* q,
                             const int32_t* block_table, const int32_t* seq_lens, int n,
                             void* out, void* stream);
