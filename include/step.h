@@ -256,7 +256,7 @@ typedef struct {
   const void* q;                      /* [n_layers_attention, n, num_q_heads, head_dim] pool dtype                */
   const void* k_new; const void* v_new; /* [n, 1, num_layers, num_kv_heads, head_dim] pool dtype                  */
   const void* hidden;                 /* [n, D] scorer dtype                                                      */
-  void* attn_out;                     /* [n_layers_attention, n, num_q_heads, head_dim] fp32                      */
+  void* attn_out;                     /* [n_layers_attention, n, num_q_heads, head_dim] fp32; must not overlap q   */
   float* step_scores_out;             /* [n] as score_steps                                                       */
   uint8_t* boundary_mask_out;         /* [n] step-end flags of the live rows (may be NULL)                        */
   float* trace_scores_out;            /* [n] score_t of every trace right after this iteration's scoring, i.e. what
