@@ -118,7 +118,7 @@ def test_random_attention_launches(seed):
     hq, hkv = [(32, 8), (8, 8), (16, 2), (40, 8), (64, 8), (4, 1), (12, 4)][int(g.integers(0, 7))]
     n = int(g.integers(1, 40))
     prefix_len = int(g.choice([0, 9, 16, 50, 160]))
-    cfg = W.scaled(W.C1, n_traces=n, num_layers=1, num_q_heads=hq, num_kv_heads=hkv, prefix_len=prefix_len, seed=11000 + seed)
+    cfg = W.scaled(W.C1, n_traces=n, num_layers=3, num_q_heads=hq, num_kv_heads=hkv, prefix_len=prefix_len, seed=11000 + seed)
     suffix = g.integers(0, int(g.choice([3, 40, 400])), size=n)
     if prefix_len == 0:
         suffix = np.maximum(suffix, 1)
@@ -139,6 +139,12 @@ def test_random_attention_launches(seed):
     got = exact_f32(tw.gpu.decode_attention(0, qd, v["block_table"][:n], v["seq_lens"][:n]))
     mx, mean = attention_errors(got, want)
     assert mx <= 1e-2 and mean <= 1e-3, ("plain", mx, mean)
+    # the three layers in one call (launches chained as programmatic dependents) = three plain calls, bit for bit
+    q3 = torch.stack([qd, qd.flip(0), qd.roll(1, 0)]).contiguous()
+    chained = tw.gpu.decode_attention_layers(0, q3, v["block_table"][:n], v["seq_lens"][:n])
+    for l in range(3):
+        assert torch.equal(chained[l], tw.gpu.decode_attention(l, q3[l], v["block_table"][:n], v["seq_lens"][:n])), ("layers", l)
+    assert np.array_equal(exact_f32(chained[0]), got)
     if hq // hkv <= 8:
         out = torch.empty((n, hq, 128), dtype=torch.float32, device="cuda:0")
         tw.gpu.decode_attention_static(0, qd, v["block_table"][:n], v["seq_lens"][:n], out)
