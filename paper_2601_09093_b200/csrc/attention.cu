@@ -773,8 +773,9 @@ extern "C" int decode_attention_shared_prefix(step_pool* pool, int layer, const 
   if (grid1 < 1) grid1 = 1;
   const int st = launch_one<kWarpsDefault, kStagesDefault, true, kPrefixPass>(p1, (int)grid1, s);
   if (st != STEP_OK) return st;
-  // pass 2
-  return launch_mma<kWarpsDefault, kStagesDefault, kSuffixPass>(pool, a, s);
+  // pass 2, a programmatic dependent of pass 1: it reads pass 1's result only where it writes its own outputs, which
+  // is behind its wait for the launch before it
+  return launch_mma<kWarpsDefault, kStagesDefault, kSuffixPass>(pool, a, s, true);
 }
 
 // =============================================================== allocation-free variant
