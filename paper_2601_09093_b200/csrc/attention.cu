@@ -21,7 +21,11 @@
 //      - a partition that holds a whole (trace, head) sequence writes the output directly;
 //        otherwise it writes an (m, l, o) partial (at most two per warp) and takes a ticket on that
 //        sequence's counter; the warp that draws the last ticket combines the sequence's partials
-//        and writes the output (no second kernel, no waiting: whoever is last does the work).
+//        and writes the output (no second kernel, no waiting: whoever is last does the work);
+//      - a launch that directly follows another launch of this kernel (the next layer of a decode step:
+//        decode_attention_layers) is made its programmatic dependent: it starts on every SM the earlier
+//        launch has left, reads and accumulates at once, and waits for that launch's completion only in
+//        front of its own first write, so the stream of KV reads does not stop at layer boundaries.
 #include "step_internal.cuh"
 
 #include <math.h>
