@@ -96,9 +96,13 @@ int kv_pool_reset(step_pool* pool, void* stream);
  * k_prefix, v_prefix: [num_layers, num_kv_heads, prefix_len, head_dim] in pool dtype.
  * Full prompt pages are allocated once and shared (refcount = n_traces); if prefix_len is
  * not a multiple of page_size every trace gets a private copy of the last, partial page.
- * Trace ids are consecutive, continuing from earlier forks; they are written to
- * trace_ids_out (HOST, n_traces ints, may be NULL).  Errors: CAPACITY, NO_BLOCKS (checked on
- * the device: the fork is then a no-op and the status word is set). */
+ * Trace ids are consecutive, continuing from the last fork that went through; they are handed out on the
+ * device.  trace_ids_out (HOST, n_traces ints, may be NULL): if given, the call synchronises the stream and
+ * writes the ids there, or -1 in every entry if the fork failed on the device; with NULL the call is
+ * asynchronous and the ids are the next n_traces in sequence.  n_traces > max_traces or a prompt longer than
+ * max_pages_per_trace pages is STEP_ERR_CAPACITY at once.  Checked on the device: more traces than max_traces
+ * in all (CAPACITY) or a free list too short (NO_BLOCKS) - the fork is then a no-op that consumes no ids and no
+ * blocks, the status word is set, and the call still returns STEP_OK. */
 int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len,
                         const void* k_prefix, const void* v_prefix,
                         int32_t* trace_ids_out, void* stream);
@@ -167,9 +171,12 @@ int decode_attention_shared_prefix(step_pool* pool, int layer, const void* q,
  *
  * Sharing: all calls on a device - from every pool and every stream - use the same array, and it
  * keeps whatever the previous call left.  The partials need no clearing (each call writes every partial
- * before it reads it); the small ticket counters in it must be zero when a call starts, which they are: they
- * start as zero bits and every call that runs to its end puts them back to zero.  Two calls that overlap in
- * time on the GPU race on the array: keep calls of this entry point ordered, e.g. on one stream. */
+ * before it reads it); the small ticket counters in it must be zero when the kernel starts, so every call
+ * clears the ones it will use (n * num_kv_heads ints) with a memset on its stream before the launch.  That
+ * also covers the one case in which a call does not leave them zero: a call whose bounded device wait ran
+ * out (STEP_ERR_TIMEOUT in the pool's status word) abandons its tickets mid-count and its outputs are
+ * undefined; the next call starts clean all the same.  Two calls that overlap in time on the GPU race on
+ * the array: keep calls of this entry point ordered, e.g. on one stream. */
 int decode_attention_static(step_pool* pool, int layer, const void* q,
                             const int32_t* block_table, const int32_t* seq_lens, int n,
                             void* out, void* stream);

@@ -213,7 +213,7 @@ class KVPool:
         ids = (C.c_int * n_traces)()
         _check("kv_pool_fork_prefix", lib().kv_pool_fork_prefix(self.handle, n_traces, prefix_len, _ptr(k_prefix),
                                                                 _ptr(v_prefix), ids, _stream(stream)))
-        return list(ids)
+        return [] if ids[0] < 0 else list(ids)           # a fork that failed on the device hands out no ids
 
     def append_kv(self, trace_ids, n_tokens, k_new, v_new, stream=None):
         _check("append_kv", lib().append_kv(self.handle, _ptr(trace_ids), trace_ids.numel(), n_tokens, _ptr(k_new),

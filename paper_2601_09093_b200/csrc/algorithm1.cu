@@ -58,13 +58,24 @@ finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, const i
   if (n_dev && *n_dev <= 0) return;      // nobody completes (every CTA reads the same count: the whole cluster leaves)
   if (cluster.block_rank() == 0) {
     const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
+    // an id listed twice completes once, at its first place in the list (v.prune_rank records that place)
+    for (int i = threadIdx.x; i < n_eff; i += blockDim.x) {
+      const int t = ids[i];
+      if (t >= 0 && t < g.max_traces) v.prune_rank[t] = 0x7fffffff;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_eff; i += blockDim.x) {
+      const int t = ids[i];
+      if (t >= 0 && t < g.max_traces) atomicMin(&v.prune_rank[t], i);
+    }
+    __syncthreads();
     int k = 0;
     for (int base = 0; base < n_eff; base += blockDim.x) {
       const int i = base + threadIdx.x;
       int t = -1, ok = 0;
       if (i < n_eff) {
         t = ids[i];
-        ok = t >= 0 && t < g.max_traces && v.live[t];
+        ok = t >= 0 && t < g.max_traces && v.live[t] && v.prune_rank[t] == i;
         if (!ok) flag_error(v.counters, STEP_ERR_BAD_TRACE);
       }
       int total;

@@ -9,8 +9,8 @@
 //  * attn_mma_kernel - bf16, head_dim 128, page 16, G <= 16.  HBM-bound design:
 //      - the whole launch's KV stream (for every trace, for every KV head, its pages in order)
 //        is cut into gridDim * kWarps equal contiguous partitions; a warp owns one partition,
-//        so all SMs finish together whatever the mix of trace lengths, and no atomics or
-//        inter-CTA waits exist;
+//        so every SM gets the same number of pages whatever the mix of trace lengths, and no CTA ever waits
+//        for another (the only atomics are the tickets of the split sequences, below);
 //      - a page of one KV head (K 4 KiB + V 4 KiB, contiguous, pre-swizzled in HBM) is brought
 //        into shared memory by ONE bulk async copy that signals an mbarrier; every warp keeps
 //        its own ring of kStages pages in flight and never synchronises with another warp;
@@ -847,19 +847,14 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   if (grid * kWarpsDefault > kStaticMaxPartitions) grid = kStaticMaxPartitions / kWarpsDefault;
   if (grid < 1) grid = 1;
   AttnArgs a;
-  a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
-  a.q = (const __nv_bfloat16*)q;
-  a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
-  a.ws_ml = scratch; a.ws_o = scratch + kStaticMlFloats; a.counters = pool->v.counters;
-  // the counters start as zero bits (static storage) and every launch leaves them zero again
+  fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
+  // the same kernel, its partials and tickets in the library's own array instead of the pool's metadata
+  a.ws_ml = scratch; a.ws_o = scratch + kStaticMlFloats;
   a.seg_cnt = reinterpret_cast<int32_t*>(scratch + kStaticMlFloats + kStaticOFloats);
-  a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
-  a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
-  const size_t smem = (size_t)kWarpsDefault * kStagesDefault * kPageBytes + (size_t)kWarpsDefault * kStagesDefault * 8 +
-                      (size_t)(n + 1) * 4;
-  auto kern = attn_mma_kernel<kWarpsDefault, kStagesDefault, false, kPlain>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
   cudaStream_t s = (cudaStream_t)stream;
-  kern<<<grid, kWarpsDefault * 32, smem, s>>>(a);
-  return launch_ok();
+  // The tickets of this call's (trace, KV head) sequences must start at zero.  A call that runs to its end leaves
+  // them zero, but one whose bounded wait ran out does not, and nothing else ever resets this array: clear them on
+  // the stream first (a memset of at most 64 KiB; no allocation).
+  STEP_CUDA_OK(cudaMemsetAsync(a.seg_cnt, 0, (size_t)n * g.Hkv * sizeof(int32_t), s));
+  return launch_one<kWarpsDefault, kStagesDefault, false, kPlain>(a, grid, s);
 }

@@ -95,19 +95,27 @@ __global__ void init_meta_kernel(DevViews v, Geo g, float unscored) {
 }
 
 // ---------------------------------------------------------------- InitTraces (fork)
-__global__ void fork_alloc_kernel(DevViews v, Geo g, int first_trace, int n_traces, int prefix_len) {
-  __shared__ int s_ok, s_fc;
+__global__ void fork_alloc_kernel(DevViews v, Geo g, int n_traces, int prefix_len) {
+  __shared__ int s_ok, s_fc, s_first;
   const int full = prefix_len / g.P, rem = prefix_len % g.P;
   const int needed = full + (rem ? n_traces : 0);
   if (threadIdx.x == 0) {
+    // trace ids are handed out here, on the device, and only by a fork that goes through: a fork that fails
+    // consumes none, so a retry after blocks were freed gets the ids the failed one would have got
+    const int first = v.counters[C_NEXT_TRACE];
+    s_first = first;
     s_fc = v.counters[C_FREE_COUNT];
-    s_ok = needed <= s_fc;
+    const bool fits = first + n_traces <= g.max_traces;
+    s_ok = fits && needed <= s_fc;
     v.counters[C_FORK_OK] = s_ok;
-    if (!s_ok) flag_error(v.counters, STEP_ERR_NO_BLOCKS);
+    v.counters[C_FORK_FIRST] = first;
+    if (!fits) flag_error(v.counters, STEP_ERR_CAPACITY);
+    else if (!s_ok) flag_error(v.counters, STEP_ERR_NO_BLOCKS);
+    if (s_ok) v.counters[C_NEXT_TRACE] = first + n_traces;
   }
   __syncthreads();
   if (!s_ok) return;
-  const int fc = s_fc;
+  const int fc = s_fc, first_trace = s_first;
   // shared full pages: pop in page order
   for (int p = threadIdx.x; p < full; p += blockDim.x) v.refcount[v.free_list[fc - 1 - p]] = n_traces;
   for (int j = 0; j < n_traces; ++j) {
@@ -135,9 +143,10 @@ __global__ void fork_alloc_kernel(DevViews v, Geo g, int first_trace, int n_trac
 // k_prefix, v_prefix: [layer, head, position, chunk].  grid (prefix_len, layer splits).
 __global__ void __launch_bounds__(256)
 fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ kpre,
-                  const uint4* __restrict__ vpre, int first_trace, int n_traces, int prefix_len, int cpr,
+                  const uint4* __restrict__ vpre, int n_traces, int prefix_len, int cpr,
                   int layers_per_cta) {
   if (!v.counters[C_FORK_OK]) return;
+  const int first_trace = v.counters[C_FORK_FIRST];
   const int pos = blockIdx.x, page = pos / g.P, slot = pos % g.P;
   const int copies = page < prefix_len / g.P ? 1 : n_traces;     // the partial page is private per trace
   const int l0 = blockIdx.y * layers_per_cta, l1 = min(g.L, l0 + layers_per_cta);
@@ -170,11 +179,23 @@ __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict
   int* s_off = sm + n;         // pops that precede this trace's
   int* s_have = sm + 2 * n;
   __shared__ int s_fc;
+  // a trace listed twice is served once, at its first place in the list; the repeats are flagged and skipped
+  // (v.prune_rank, scratch of max_traces ints, records the first place that names each trace)
+  for (int i = threadIdx.x; i < n_eff; i += blockDim.x) {
+    const int t = ids[i];
+    if (t >= 0 && t < g.max_traces) v.prune_rank[t] = 0x7fffffff;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_eff; i += blockDim.x) {
+    const int t = ids[i];
+    if (t >= 0 && t < g.max_traces) atomicMin(&v.prune_rank[t], i);
+  }
+  __syncthreads();
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     int need = -1, have = 0;
     if (i >= n_eff) { s_need[i] = need; s_have[i] = have; continue; }
     const int t = ids[i];
-    if (t < 0 || t >= g.max_traces || !v.live[t]) {
+    if (t < 0 || t >= g.max_traces || !v.live[t] || v.prune_rank[t] != i) {
       flag_error(v.counters, STEP_ERR_BAD_TRACE);
     } else {
       const int S = v.seq_lens[t];
@@ -315,7 +336,6 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->elem_bytes = cfg->dtype == STEP_BF16 ? 2 : 4;
   p->swizzle = (cfg->dtype == STEP_BF16 && cfg->head_dim % 64 == 0) ? 1 : 0;
   p->max_score_rows = cfg->max_score_rows > 0 ? cfg->max_score_rows : cfg->max_traces;
-  p->next_trace = 0;
   p->num_sms = sms;
   p->attn_grid = sms;
   p->fast_path = 1;
@@ -362,7 +382,6 @@ int kv_pool_reset(step_pool* pool, void* stream) {
   size_t items = (size_t)g.max_traces * g.max_pages;
   if ((size_t)g.num_blocks > items) items = g.num_blocks;
   init_meta_kernel<<<grid_for(items, 256, pool->num_sms), 256, 0, (cudaStream_t)stream>>>(pool->v, g, pool->cfg.unscored_score);
-  pool->next_trace = 0;
   return launch_ok();
 }
 
@@ -371,11 +390,10 @@ int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const voi
   if (!pool || n_traces < 1 || prefix_len < 0) return STEP_ERR_INVALID_ARG;
   if (prefix_len > 0 && (!k_prefix || !v_prefix)) return STEP_ERR_INVALID_ARG;
   Geo g = geo_of(pool);
-  if (pool->next_trace + n_traces > g.max_traces) return STEP_ERR_CAPACITY;
+  if (n_traces > g.max_traces) return STEP_ERR_CAPACITY;
   if ((prefix_len + g.P - 1) / g.P > g.max_pages) return STEP_ERR_CAPACITY;
-  const int first = pool->next_trace;
   cudaStream_t s = (cudaStream_t)stream;
-  fork_alloc_kernel<<<1, 256, 0, s>>>(pool->v, g, first, n_traces, prefix_len);
+  fork_alloc_kernel<<<1, 256, 0, s>>>(pool->v, g, n_traces, prefix_len);
   if (prefix_len > 0) {
     const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
     int splits = (2 * pool->num_sms + prefix_len - 1) / prefix_len;
@@ -384,12 +402,17 @@ int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const voi
     const int layers_per_cta = (g.L + splits - 1) / splits;
     splits = (g.L + layers_per_cta - 1) / layers_per_cta;
     fork_write_kernel<<<dim3((unsigned)prefix_len, (unsigned)splits), 256, 0, s>>>(
-        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_prefix, (const uint4*)v_prefix, first,
+        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_prefix, (const uint4*)v_prefix,
         n_traces, prefix_len, cpr, layers_per_cta);
   }
-  pool->next_trace += n_traces;
-  if (trace_ids_out) for (int j = 0; j < n_traces; ++j) trace_ids_out[j] = first + j;
-  return launch_ok();
+  const int st = launch_ok();
+  if (st != STEP_OK || !trace_ids_out) return st;
+  // the ids were decided on the device: fetch the outcome (the one synchronising path of this call)
+  int32_t h[C_FORK_FIRST + 1];
+  STEP_CUDA_OK(cudaMemcpyAsync(h, pool->v.counters, sizeof(h), cudaMemcpyDeviceToHost, s));
+  STEP_CUDA_OK(cudaStreamSynchronize(s));
+  for (int j = 0; j < n_traces; ++j) trace_ids_out[j] = h[C_FORK_OK] ? h[C_FORK_FIRST] + j : -1;
+  return STEP_OK;
 }
 
 int append_kv(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,

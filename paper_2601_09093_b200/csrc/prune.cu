@@ -95,16 +95,25 @@ release_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, float 
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ int s_warp[33];
-  // keep the valid, live ids in the order given
-  if (cluster.block_rank() == 0 && threadIdx.x == 0) {
-    int k = 0;
-    for (int i = 0; i < n; ++i) {
+  // keep the valid, live ids in the order given; an id listed twice is released once (at its first place) and the
+  // repeat flagged - counting it twice would take two references off every one of its blocks
+  if (cluster.block_rank() == 0) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
       const int t = ids[i];
-      if (t < 0 || t >= g.max_traces || !v.live[t]) { flag_error(v.counters, STEP_ERR_BAD_TRACE); continue; }
-      v.prune_list[k++] = t;
+      if (t >= 0 && t < g.max_traces) v.prune_rank[t] = 0;
     }
-    v.counters[C_PRUNE_N] = k;
-    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int k = 0;
+      for (int i = 0; i < n; ++i) {
+        const int t = ids[i];
+        if (t < 0 || t >= g.max_traces || !v.live[t] || v.prune_rank[t]) { flag_error(v.counters, STEP_ERR_BAD_TRACE); continue; }
+        v.prune_rank[t] = 1;
+        v.prune_list[k++] = t;
+      }
+      v.counters[C_PRUNE_N] = k;
+      __threadfence();
+    }
   }
   cluster.sync();
   release_listed_cluster(v, g, __ldcg(&v.counters[C_PRUNE_N]), unscored, s_warp);

@@ -33,6 +33,8 @@ enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_
                // Algorithm 1 driver: live / finishing traces of the current iteration, running totals
                C_IT_NLIVE = 8, C_IT_NFIN = 9, C_N_FINISHED = 10, C_N_EVICTED = 11, C_IT_NPRUNED = 12,
                C_SCORE_TILE = 13,   // rows per work item of the tensor-core scorer kernel (128 or 256)
+               C_NEXT_TRACE = 14,   // id the next successful fork starts at
+               C_FORK_FIRST = 15,   // first id of the most recent fork (valid when C_FORK_OK is set)
                C_NUM = 64 };
 
 struct MetaLayout {
@@ -67,7 +69,6 @@ struct step_pool {
   int elem_bytes;
   int swizzle;        // 1: rows stored with XOR-swizzled 16-byte chunks
   int max_score_rows;
-  int next_trace;     // host-side id allocator for forks
   int num_sms;
   int attn_grid;      // CTAs of the tensor-core attention launch
   int fast_path;      // 1 allowed, -1 forced off

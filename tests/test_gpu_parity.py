@@ -113,6 +113,60 @@ def test_error_conditions_are_flagged_not_fatal():
     assert tw3.gpu.last_error()[1] == 1 << 2 and tw3.gpu.stats() == dict(used=0, free=1, total=1, live_traces=0)
 
 
+def test_a_fork_that_fails_consumes_no_ids_and_can_be_retried():
+    """Row i of the loop's inputs is trace i, so ids must not be lost to a fork the pool could not serve: the retry
+    after blocks were freed gets the ids the failed fork would have got - as in the oracle."""
+    cfg = W.scaled(W.C0, prefix_len=0)
+    tw = Twin(cfg, 6, 4, 4, store_payload=False)
+    ids, oids = tw.fork(2, 40)                                   # 2 shared pages + a private partial page each: 4 blocks
+    assert ids == oids == [0, 1]
+    ids, oids = tw.fork(2, 40)                                   # needs 4 more, 2 are free
+    assert ids == oids == []
+    assert tw.status() == (1 << 2, 1 << 2)
+    tw.assert_meta_equal()
+    tw.gpu.release_traces(torch.tensor([0, 1], dtype=torch.int32, device="cuda"))
+    tw.ora.release_trace(0); tw.ora.release_trace(1)
+    ids, oids = tw.fork(2, 40)                                   # now it fits, and takes ids 2 and 3 on both sides
+    assert ids == oids == [2, 3]
+    assert tw.append(ids, 8) == [True, True]
+    tw.assert_meta_equal()
+    ids, oids = tw.fork(1, 16)                                   # a fifth trace in a pool of four
+    assert ids == oids == []
+    assert tw.status() == (1 << 4, 1 << 4)
+    tw.assert_meta_equal()
+    tw.gpu.reset(); torch.cuda.synchronize()
+    assert tw.gpu.fork_prefix(1, 0, None, None) == [0]           # a reset pool starts again at id 0
+
+
+def test_an_id_listed_twice_is_served_once_and_flagged():
+    """append_kv, kv_pool_release_traces and kv_pool_finish_traces take lists of distinct ids; a repeat is flagged
+    (BAD_TRACE) and skipped, so the pool ends as if the list had named the trace once at its first place."""
+    cfg = W.scaled(W.C0, prefix_len=32)
+    tw = Twin(cfg, 64, 8, 6, store_payload=False)
+    ids, _ = tw.fork(6, 32)
+    dev = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+    z = torch.zeros((7, 20, 1, 1, 64), device="cuda")
+    tw.gpu.append_kv(dev([3, 1, 3, 5, 1, 3, 0]), 20, z, z)
+    assert tw.ora.append_kv([3, 1, 5, 0], 20) == [True] * 4
+    tw.assert_meta_equal()
+    assert tw.gpu.last_error()[1] == 1 << 3
+    tw.gpu.release_traces(dev([4, 1, 4, 1]))
+    tw.ora.release_trace(4); tw.ora.release_trace(1)
+    tw.assert_meta_equal()
+    assert tw.gpu.last_error()[1] == 1 << 3
+    tw.gpu.finish_traces(dev([5, 0, 5]), dev([7, 8, 9]))
+    tw.ora.release_trace(5); tw.ora.release_trace(0)
+    tw.assert_meta_equal()
+    assert tw.gpu.last_error()[1] == 1 << 3
+    vv = tw.gpu.vote_views()
+    assert vv["answer"][5].item() == 7 and vv["answer"][0].item() == 8
+    assert tw.gpu.stats()["live_traces"] == 2                    # traces 2 and 3; the shared prompt pages are still theirs
+    tw.gpu.release_traces(dev([2, 3, 2]))
+    tw.ora.release_trace(2); tw.ora.release_trace(3)
+    tw.assert_meta_equal()
+    assert tw.gpu.stats()["used"] == 0
+
+
 def test_host_side_argument_checks():
     pool = H.make_pool(W.C0, 8, 4)
     z = torch.zeros(4, device="cuda")

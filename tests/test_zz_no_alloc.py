@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import attention as OA
 from paper_2601_09093_b200 import binding as B
 from paper_2601_09093_b200 import harness as H
 from paper_2601_09093_b200 import workloads as W
@@ -55,6 +56,64 @@ def test_static_scratch_matches_regular_entry_point_twice_in_a_row():
     # and a different pool on the same device shares the same array
     pool2 = _pool_with_traces(W.scaled(W.C1, n_traces=3, prefix_len=16, num_q_heads=64), [700, 20, 1500], seed=12)
     _compare(pool2, W.scaled(W.C1, n_traces=3, prefix_len=16, num_q_heads=64), 3, q_sub=3)
+
+
+def test_static_call_allocates_nothing_and_agrees_with_the_oracle():
+    """What the entry point is for: after the first call on the device (which looks up the array's address) a
+    call leaves the driver's free memory and torch's allocator exactly as it found them.  The result of that
+    call is also compared with the CPU oracle directly, on K/V rows read back from the pool."""
+    cfg = W.scaled(W.C1, n_traces=5, prefix_len=32)
+    suffix = [3, 700, 0, 1900, 65]
+    pool = _pool_with_traces(cfg, suffix, seed=21)
+    v = pool.views()
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (5, cfg.num_q_heads, cfg.head_dim), "bf16", sub=9)
+    q = H.to_device(qb, "bf16")
+    out = torch.empty((5, cfg.num_q_heads, cfg.head_dim), dtype=torch.float32, device="cuda")
+    bt, sl = v["block_table"][:5], v["seq_lens"][:5]
+    pool.decode_attention_static(0, q, bt, sl, out)              # first call on this device: set-up included
+    torch.cuda.synchronize()
+    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    out.fill_(float("nan"))
+    pool.decode_attention_static(0, q, bt, sl, out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    got = out.cpu().numpy().astype(np.float64)
+    for t in range(5):
+        S = cfg.prefix_len + suffix[t]
+        K_ = np.empty((S, cfg.num_kv_heads, cfg.head_dim)); V_ = np.empty_like(K_)
+        for h in range(cfg.num_kv_heads):
+            k, vv = pool.read_kv(0, h, v["block_table"][t], S)
+            K_[:, h] = k.float().cpu().numpy(); V_[:, h] = vv.float().cpu().numpy()
+        err = np.abs(got[t] - OA.dense_decode_attention(qx[t].astype(np.float64), K_, V_))
+        assert err.max() <= ATT_MAX and err.mean() <= ATT_MEAN
+    assert pool.last_error() == (0, 0)
+
+
+def test_static_scratch_rejects_more_sequences_than_its_counters_hold():
+    """n > 2048 traces, or more than 16,384 (trace, KV head) sequences, do not fit the fixed array: STEP_ERR_CAPACITY
+    before anything is launched, the output untouched."""
+    one_head = W.scaled(W.C1, n_traces=2049, prefix_len=0, num_q_heads=4, num_kv_heads=1)
+    pool = H.make_pool(one_head, 8, 2, 2049)
+    v = pool.views()
+    q = torch.zeros((2049, 4, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.full((2049, 4, 128), 7.0, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.StepError) as e:
+        pool.decode_attention_static(0, q, v["block_table"], v["seq_lens"], out)
+    assert e.value.code == 4
+    many_heads = W.scaled(W.C1, n_traces=1100, prefix_len=0, num_q_heads=16, num_kv_heads=16)     # 17,600 sequences
+    pool2 = H.make_pool(many_heads, 8, 2, 1100)
+    v2 = pool2.views()
+    q2 = torch.zeros((1100, 16, 128), dtype=torch.bfloat16, device="cuda")
+    out2 = torch.full((1100, 16, 128), 7.0, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.StepError) as e:
+        pool2.decode_attention_static(0, q2, v2["block_table"], v2["seq_lens"], out2)
+    assert e.value.code == 4
+    torch.cuda.synchronize()
+    assert (out == 7.0).all() and (out2 == 7.0).all()
+    pool2.decode_attention_static(0, q2[:1024], v2["block_table"][:1024], v2["seq_lens"][:1024], out2[:1024])   # 16,384: fits
+    torch.cuda.synchronize()
+    assert (out2[:1024] == 0.0).all()                            # empty traces give zeros
 
 
 def test_static_scratch_rejects_what_does_not_fit():
