@@ -137,6 +137,21 @@ int decode_attention_layers(step_pool* pool, int layer0, int n_layers, const voi
                             const int32_t* block_table, const int32_t* seq_lens, int n,
                             void* out, void* stream);
 
+/* decode_attention for a caller that runs the model layer by layer (the attention inside NextToken of Algorithm 1: the
+ * query of layer l + 1 is computed from the output of layer l, so the queries of all layers are never at hand
+ * together and decode_attention_layers does not apply).  Same arguments and the same result, bit for bit, as
+ * decode_attention.  The launch is made a programmatic dependent of whatever kernel directly precedes it in the
+ * stream - meant to be the caller's kernel that writes q: its CTAs are scheduled while that kernel is finishing, work
+ * out their shares from seq_lens, start their first page copies through block_table, and wait for that kernel's
+ * completion (and with it for everything earlier in the stream) only in front of their first read of q.
+ * Requirement: the kernel directly before this call in the stream must not write seq_lens, block_table or this
+ * layer's cache (do not issue it directly after append_kv or a prune), and it must itself be ordered after
+ * everything before it, as any kernel launched the ordinary way is.  Shapes the tensor-core kernel does not cover
+ * are launched the ordinary way. */
+int decode_attention_dependent(step_pool* pool, int layer, const void* q,
+                               const int32_t* block_table, const int32_t* seq_lens, int n,
+                               void* out, void* stream);
+
 /* decode_attention for traces that share their first pages (the prompt pages kv_pool_fork_prefix allocates once for
  * all traces of a problem: Algorithm 1, InitTraces):
  *   out[i] = attention of q[i] over the prefix_pages * page_size positions stored in blocks prefix_blocks[0 ..
@@ -379,6 +394,15 @@ int kv_pool_set_scorer_config(step_pool* pool, int mode, int tc_min_rows);
  * *n_rows = boundary rows it found, *tc_units = hidden units per CTA of the tensor-core kernel, or 0 if
  * the CUDA-core kernel scored the rows.  Host ints, either may be NULL; synchronises the stream. */
 int kv_pool_score_launch_info(step_pool* pool, int* n_rows, int* tc_units, void* stream);
+/* Measurement aid (the paper has no counterpart): the rate at which this device's HBM feeds the copy structure of
+ * decode_attention when no arithmetic is attached - one CTA per SM, eight warps, each streaming an equal
+ * contiguous share of buf through a ring of three 8 KiB bulk copies into shared memory and dropping the data.
+ * n_launches launches over the same buffer; chained != 0 makes every launch after the first a programmatic
+ * dependent of the one before it, as decode_attention_layers does with its layers.  buf: device, 16-byte aligned,
+ * bytes >= 8192 (a multiple of 8192 is read); err_flag: [1] int32 device, set to 1 if a bounded wait ran out.
+ * Asynchronous on the stream; time it with events around the call. */
+int step_read_stream_probe(const void* buf, size_t bytes, int n_launches, int chained, int32_t* err_flag,
+                           void* stream);
 /* Library build tag, for logs. */
 const char* step_version(void);
 

@@ -93,6 +93,8 @@ def lib():
     L.append_kv.argtypes = [vp, vp, i, i, vp, vp, vp]
     L.decode_attention.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_static.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.decode_attention_dependent.argtypes = [vp, i, vp, vp, vp, i, vp, vp]
+    L.step_read_stream_probe.argtypes = [vp, C.c_size_t, i, i, vp, vp]
     L.decode_attention_layers.argtypes = [vp, i, i, vp, vp, vp, i, vp, vp]
     L.decode_attention_shared_prefix.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
     L.score_steps.argtypes = [vp, vp, vp, vp, i, C.POINTER(scorer_weights), vp, vp]
@@ -225,6 +227,16 @@ class KVPool:
             out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
         _check("decode_attention", lib().decode_attention(self.handle, layer, _ptr(q), _ptr(block_table), _ptr(seq_lens),
                                                           n, _ptr(out), _stream(stream)))
+        return out
+
+    def decode_attention_dependent(self, layer, q, block_table, seq_lens, out=None, stream=None):
+        """decode_attention launched as a programmatic dependent of the kernel that precedes it in the stream (the one
+        that writes q)."""
+        n = q.shape[0]
+        if out is None:
+            out = torch.empty((n, self.num_q_heads, self.head_dim), dtype=torch.float32, device=q.device)
+        _check("decode_attention_dependent", lib().decode_attention_dependent(self.handle, layer, _ptr(q), _ptr(block_table),
+                                                                              _ptr(seq_lens), n, _ptr(out), _stream(stream)))
         return out
 
     def decode_attention_layers(self, layer0, q, block_table, seq_lens, out=None, stream=None):
@@ -406,6 +418,12 @@ class ScorerTrainer:
             self.D, self.m, _ptr(self.adam_m), _ptr(self.adam_v), C.byref(self.h), _ptr(self.ws), self.ws_bytes,
             _ptr(self.loss), _stream(stream)))
         return self.loss
+
+
+def read_stream_probe(buf, n_launches, chained, err_flag, stream=None):
+    """step_read_stream_probe over the bytes of `buf` (a contiguous device tensor); no sync."""
+    _check("step_read_stream_probe", lib().step_read_stream_probe(_ptr(buf), buf.numel() * buf.element_size(), n_launches,
+                                                                  int(bool(chained)), _ptr(err_flag), _stream(stream)))
 
 
 def step_end_table_from_vocab(token_texts):

@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstep.so")
 STAMP = os.path.join(HERE, "_build", "libstep.stamp")
-SOURCES = ["pool.cu", "attention.cu", "scorer.cu", "scorer_tc.cu", "prune.cu", "algorithm1.cu", "train.cu"]
+SOURCES = ["pool.cu", "attention.cu", "scorer.cu", "scorer_tc.cu", "prune.cu", "algorithm1.cu", "train.cu", "probe.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "--use_fast_math", "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v"]
 

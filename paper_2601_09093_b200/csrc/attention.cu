@@ -27,6 +27,7 @@
 //        launch has left, reads and accumulates at once, and waits for that launch's completion only in
 //        front of its own first write, so the stream of KV reads does not stop at layer boundaries.
 #include "step_internal.cuh"
+#include "async_copy.cuh"
 
 #include <math.h>
 
@@ -114,7 +115,6 @@ attn_scalar_kernel(Geo g, const T* __restrict__ kv, int layer, const T* __restri
 constexpr int kP = 16, kD = 128;
 constexpr int kPageBytes = 2 * kP * kD * 2;        // K rows then V rows of one KV head: 8 KiB
 constexpr int kVOffset = kP * kD * 2;              // 4 KiB
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a bounded wait gives up after 2 s
 
 struct AttnArgs {
   const __nv_bfloat16* kv_layer;   // kv_storage + layer offset
@@ -134,6 +134,7 @@ struct AttnArgs {
   float* pre_o;                    // [n][Hq][kD] its weighted value sum
   int pp;                          // shared pages
   int tpb, n_bundles;              // prefix pass: traces per 16-row bundle of query rows, number of bundles
+  int q_from_primary;              // 1: the launch before this one in the stream writes q (see decode_attention_dependent)
 };
 
 // kMode of attn_mma_kernel: the plain kernel; the pass over the shared pages, whose 16 query rows are the G heads of
@@ -141,44 +142,6 @@ struct AttnArgs {
 // (trace, head) in pre_ml / pre_o; and the pass over every trace's own pages, which folds that result in at the end.
 constexpr int kPlain = 0, kPrefixPass = 1, kSuffixPass = 2;
 
-__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ inline unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Waits for the phase with the given parity; false if the time limit ran out.
-__device__ inline bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > kWaitLimitNs) return false;
-  }
-}
-// One page: global (16-byte aligned) -> shared, completion counted in bytes on the mbarrier.
-__device__ inline void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 __device__ inline void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -270,8 +233,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   }
   if (lane == 0) {
     for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&s_bar[warp * kStages + s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_init_fence();
   }
   __syncthreads();
 
@@ -279,6 +241,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   // launch was scheduled ahead of the completion of such a launch before it (a layer-by-layer sequence of calls made
   // by the library itself), it may run up to its first write - of an output, a partial or a ticket - and must then
   // wait for that launch, whose partials and tickets share the scratch.  A no-op for a launch made the plain way.
+  // When the launch before this one is the caller's own kernel that produces q (q_from_primary), the wait moves up to
+  // the first read of q: what precedes it - the prefix sums above, the barriers, and every warp's first kStages page
+  // copies - depends only on the lengths, the block table and the cache, and overlaps that kernel's tail.
   dependents_may_launch();
   bool waited = false;
   auto before_first_write = [&]() { if (!waited) { wait_for_primary(); waited = true; } };
@@ -363,6 +328,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   for (int i = 0; i < cnt; ++i) {
     if (!seg_open) {
       // new (trace, head) segment: Q fragments of the G heads of this group, fresh softmax state
+      if (a.q_from_primary) before_first_write();
       const uint32_t *q0, *q1;
       bool r0, r1;
       if constexpr (kMode == kPrefixPass) {
@@ -683,6 +649,7 @@ void fill_args(AttnArgs& a, const step_pool* pool, const Geo& g, int layer, cons
   a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
   a.prefix_blocks = nullptr; a.pre_ml = nullptr; a.pre_o = nullptr; a.pp = 0; a.tpb = 1; a.n_bundles = 0;
+  a.q_from_primary = 0;
 }
 
 bool mma_shape(const step_pool* pool, const Geo& g, int n) {
@@ -691,12 +658,27 @@ bool mma_shape(const step_pool* pool, const Geo& g, int n) {
 
 }  // namespace
 
+// How a launch relates to the kernel before it in the stream: an ordinary launch; a programmatic dependent of
+// another launch of this kernel on the same pool (waits in front of its first write); a programmatic dependent of
+// the caller's kernel that writes q (waits in front of its first read of q).
+enum LaunchMode { kOrdinary = 0, kAfterOwnKind = 1, kAfterQProducer = 2 };
+
 static int decode_attention_launch(step_pool* pool, int layer, const void* q, const int32_t* block_table,
-                                   const int32_t* seq_lens, int n, void* out, void* stream, bool dependent);
+                                   const int32_t* seq_lens, int n, void* out, void* stream, LaunchMode mode);
 
 extern "C" int decode_attention(step_pool* pool, int layer, const void* q, const int32_t* block_table,
                                 const int32_t* seq_lens, int n, void* out, void* stream) {
-  return decode_attention_launch(pool, layer, q, block_table, seq_lens, n, out, stream, false);
+  return decode_attention_launch(pool, layer, q, block_table, seq_lens, n, out, stream, kOrdinary);
+}
+
+// decode_attention for a caller that runs the layers one by one (the query of layer l + 1 is computed from the
+// output of layer l, so it cannot hand over all layers' queries at once): the launch is made a programmatic dependent
+// of whatever kernel precedes it in the stream - the caller's kernel that produces q.  The CTAs are scheduled as
+// soon as that kernel's CTAs have exited (or have announced that dependents may start), set themselves up, start
+// their first page copies, and wait for that kernel's completion only in front of their first read of q.
+extern "C" int decode_attention_dependent(step_pool* pool, int layer, const void* q, const int32_t* block_table,
+                                          const int32_t* seq_lens, int n, void* out, void* stream) {
+  return decode_attention_launch(pool, layer, q, block_table, seq_lens, n, out, stream, kAfterQProducer);
 }
 
 // decode_attention of several consecutive layers whose queries the caller has at hand.  The first layer's launch is an
@@ -714,14 +696,14 @@ extern "C" int decode_attention_layers(step_pool* pool, int layer0, int n_layers
   const size_t o_layer = (size_t)n * pool->cfg.num_q_heads * pool->cfg.head_dim * sizeof(float);
   for (int l = 0; l < n_layers; ++l) {
     const int st = decode_attention_launch(pool, layer0 + l, q ? (const char*)q + l * q_layer : nullptr, block_table, seq_lens, n,
-                                           out ? (char*)out + l * o_layer : nullptr, stream, l > 0);
+                                           out ? (char*)out + l * o_layer : nullptr, stream, l > 0 ? kAfterOwnKind : kOrdinary);
     if (st != STEP_OK) return st;
   }
   return STEP_OK;
 }
 
 static int decode_attention_launch(step_pool* pool, int layer, const void* q, const int32_t* block_table,
-                                   const int32_t* seq_lens, int n, void* out, void* stream, bool dependent) {
+                                   const int32_t* seq_lens, int n, void* out, void* stream, LaunchMode mode) {
   if (!pool || n < 0) return STEP_ERR_INVALID_ARG;
   if (n == 0) return STEP_OK;
   if (!q || !block_table || !seq_lens || !out) return STEP_ERR_INVALID_ARG;
@@ -731,8 +713,10 @@ static int decode_attention_launch(step_pool* pool, int layer, const void* q, co
   if (pool->fast_path > 0 && mma_shape(pool, g, n)) {
     AttnArgs a;
     fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
-    return launch_mma<kWarpsDefault, kStagesDefault, kPlain>(pool, a, s, dependent);
+    a.q_from_primary = mode == kAfterQProducer;
+    return launch_mma<kWarpsDefault, kStagesDefault, kPlain>(pool, a, s, mode != kOrdinary);
   }
+  // the scalar kernel is always launched the ordinary way (same results, no overlap)
   if (n > 65535) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)(g.d + kScalarWarps * g.d) * sizeof(float);
   if (pool->cfg.dtype == STEP_BF16)

@@ -16,6 +16,7 @@
 //             scores are folded into its (sum, count) in ascending row order (per 512-row CTA, the
 //             CTA partials in CTA order) and the mean is refreshed.
 #include "step_internal.cuh"
+#include "block_scan.cuh"
 
 #include <cooperative_groups.h>
 #include <math.h>
@@ -57,34 +58,6 @@ __device__ inline bool row_flag(const FlagSource& f, int i, int32_t* counters) {
   return e;
 }
 
-// Block-wide exclusive prefix sum of one int per thread; *total gets the sum.
-__device__ inline int compact_scan(int x, int* s_warp, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = x;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  __syncthreads();
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const int w = s_warp[lane];
-    int wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    s_warp[lane] = wi - w;
-    if (lane == 31) s_warp[32] = wi;
-  }
-  __syncthreads();
-  *total = s_warp[32];
-  return s_warp[warp] + incl - x;
-}
-
 // A cluster of kCompactCtas CTAs; CTA r owns the r-th contiguous share of the rows.  Pass 1 counts the step-end
 // rows of the share, the counts are exchanged through distributed shared memory, pass 2 writes the row list
 // (ascending over the whole launch) and NaN into the other rows.
@@ -117,7 +90,7 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
   }
   {
     int total;
-    compact_scan(mine, s_warp, &total);
+    block_excl_scan(mine, s_warp, &total);
     if (threadIdx.x == 0) s_count = total;
   }
   cluster.sync();
@@ -143,7 +116,7 @@ score_compact_kernel(DevViews v, FlagSource src, int M, float* __restrict__ step
         if (i0 + j < hi && row_flag(src, i0 + j, v.counters)) flags |= 1u << j;
     }
     int total;
-    int at = running + compact_scan(__popc(flags), s_warp, &total);
+    int at = running + block_excl_scan(__popc(flags), s_warp, &total);
 #pragma unroll
     for (int j = 0; j < kRowsPerThread; ++j) {
       if (flags & (1u << j)) v.score_idx[at++] = i0 + j;

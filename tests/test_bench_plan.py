@@ -14,7 +14,7 @@ from paper_2601_09093_b200 import workloads as W  # noqa: E402
 
 @pytest.mark.parametrize("traces,threshold", [(0, 0.0), (16, 0.0), (32, 0.5), (32, 0.9)])
 def test_memory_saturated_plan_stays_below_the_trigger_during_the_timed_steps(traces, threshold):
-    steps_total = 3 + 10 + 13 + 4 + bench.ALG1_ITERATIONS + 3 + bench.ALG1_GRAPH_ITERATIONS + 2      # as run_ours counts them
+    steps_total = bench.planned_steps(10, 3, 10)                    # as run_ours counts them
     cfg, suffix, nb, max_pages, layers = bench.workload_plan("c3", 0, steps_total, None, traces, threshold)
     T, P = cfg.n_traces, cfg.page_size
     assert T == (traces or 64) and layers == 36 and nb == 65536

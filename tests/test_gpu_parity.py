@@ -145,8 +145,8 @@ def test_an_id_listed_twice_is_served_once_and_flagged():
     tw = Twin(cfg, 64, 8, 6, store_payload=False)
     ids, _ = tw.fork(6, 32)
     dev = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
-    z = torch.zeros((7, 20, 1, 1, 64), device="cuda")
-    tw.gpu.append_kv(dev([3, 1, 3, 5, 1, 3, 0]), 20, z, z)
+    z = torch.zeros((6, 20, 1, 1, 64), device="cuda")
+    tw.gpu.append_kv(dev([3, 1, 3, 5, 1, 0]), 20, z, z)           # (a list may not be longer than max_traces)
     assert tw.ora.append_kv([3, 1, 5, 0], 20) == [True] * 4
     tw.assert_meta_equal()
     assert tw.gpu.last_error()[1] == 1 << 3
@@ -506,3 +506,49 @@ def test_attention_layers_call_equals_layer_by_layer_calls(hq, hkv):
     assert tw.status() == (0, 0)
     with pytest.raises(B.StepError):
         tw.gpu.decode_attention_layers(3, qd[:3], v["block_table"][:9], v["seq_lens"][:9])     # layers 3, 4, 5: one too many
+
+
+@pytest.mark.parametrize("grid", [148, 5])
+def test_dependent_launch_waits_for_the_kernel_that_writes_q(grid):
+    """decode_attention_dependent is scheduled while the kernel before it - here a 256 MB copy whose first rows are
+    the queries - is still running, and must not read q before that kernel has completed: the buffer holds NaN bit
+    patterns until the copy lands.  Results equal the plain call's, bit for bit, layer after layer."""
+    cfg = W.scaled(W.C1, n_traces=9, num_layers=3, prefix_len=40, seed=818)
+    tw, ids = _build(cfg, [0, 300, 17, 1200, 64, 5, 900, 33, 2000])
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (3, 9, 32, 128), "bf16")
+    qd = H.to_device(qb, "bf16")
+    v = tw.gpu.views()
+    tw.gpu.set_attention_config(grid_ctas=grid)
+    n_q = 9 * 32 * 128
+    big_src = torch.zeros(128 << 20, dtype=torch.bfloat16, device="cuda")
+    big_dst = torch.empty_like(big_src)
+    for rep in range(3):
+        for l in range(3):
+            big_dst.view(torch.int16).fill_(0x7FC0)              # NaN everywhere, the query rows included
+            big_src[:n_q] = qd[l].reshape(-1)
+            torch.mul(big_src, 1, out=big_dst)                   # the kernel that "produces" q (an elementwise kernel, not a memcpy)
+            got = tw.gpu.decode_attention_dependent(l, big_dst[:n_q].view(9, 32, 128), v["block_table"][:9], v["seq_lens"][:9])
+            one = tw.gpu.decode_attention(l, qd[l], v["block_table"][:9], v["seq_lens"][:9])
+            assert torch.equal(got, one), (rep, l)
+    want = _oracle_attention(tw, 2, qx[2], 9)
+    mx, mean = attention_errors(exact_f32(got), want)
+    assert mx <= ATT_MAX and mean <= ATT_MEAN
+    assert tw.status() == (0, 0)
+    # a pool the tensor-core kernel does not cover takes the ordinary launch
+    tw0, _ = _build(W.C0, [5, 40])
+    q0b, q0x = W.normal(W.C0.seed, W.TID_Q, (2, 4, 64), "fp32")
+    v0 = tw0.gpu.views()
+    a = tw0.gpu.decode_attention_dependent(0, H.to_device(q0b, "fp32"), v0["block_table"][:2], v0["seq_lens"][:2])
+    b = tw0.gpu.decode_attention(0, H.to_device(q0b, "fp32"), v0["block_table"][:2], v0["seq_lens"][:2])
+    assert torch.equal(a, b)
+
+
+def test_read_stream_probe_runs_clean_both_ways():
+    buf = torch.empty((64 << 20) + 4096, dtype=torch.uint8, device="cuda")      # not a whole number of 8 KiB pieces
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for chained in (0, 1):
+        B.read_stream_probe(buf, 5, chained, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    with pytest.raises(B.StepError):
+        B.read_stream_probe(buf[:4096], 1, 0, err)
