@@ -177,7 +177,7 @@ def workload_plan(name, num_blocks_override, steps_total, free_bytes=None, trace
 def planned_steps(K, Wm, e2e_steps):
     """Tokens every trace gains over a whole default run (timed steps, the per-layer-call legs, the end-to-end leg, the
     library-driven loop): the state is sized so that the trigger stays quiet through all of them."""
-    return Wm + K + 3 * (2 + K) + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS + 3 + ALG1_GRAPH_ITERATIONS + 2
+    return Wm + K + 3 * (2 + K) + (Wm + e2e_steps) + 4 + ALG1_ITERATIONS_ONE_LAYER + 3 + ALG1_GRAPH_ITERATIONS + 2
 
 
 def run_ours(args):
@@ -225,6 +225,9 @@ def run_ours(args):
         return torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
     sets = []
     mask_np = [W.boundary_mask(cfg, T, sub=100 + i) for i in range(NSETS)]
+    for i, mk in enumerate(mask_np):
+        if not mk.any():
+            mk[i % T] = 1                # every timed step scores at least one step end (the expected number per step is one or two)
     for i in range(NSETS):
         s = dict(q=rnd(L, T, cfg.num_q_heads, cfg.head_dim), k=rnd(T, 1, phys_layers, cfg.num_kv_heads, cfg.head_dim),
                  v=rnd(T, 1, phys_layers, cfg.num_kv_heads, cfg.head_dim), h=rnd(T, cfg.scorer_D),
@@ -473,7 +476,7 @@ def run_ours(args):
         # the same launches counted the way a per-trace kernel would see them (the shared prompt once per trace)
         "kv_gbs_logical": float(np.sum(seq_now - K // 2)) * cfg.bytes_per_token_layer / (attn_avg_ms * 1e-3) / 1e9,
         "attention_share_of_step": float(np.sum(attn_run_ms)) / ms_total,
-        "gpu_launches": K * (2 + L + 3 + 1), "clocks": clocks,
+        "gpu_launches": K * (2 + L + 1 + 1), "clocks": clocks,
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
     if e2e:
@@ -600,7 +603,8 @@ def cpu_baseline_and_parity(pool, cfg, s, out, L, phys_layers, cpu_budget_s=12.0
 
 
 # ---------------------------------------------------------------------------------------------
-ALG1_ITERATIONS = 6
+ALG1_ITERATIONS = 6                 # iterations of the directly launched run on the 36-layer workloads
+ALG1_ITERATIONS_ONE_LAYER = 40      # ... and on the one-layer workloads, where the end-of-call round trip would weigh on six
 ALG1_GRAPH_ITERATIONS = 40          # iterations of the recorded-iteration run on the one-layer workloads (6 on the others)
 
 
@@ -614,8 +618,9 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     vocab = W.synthetic_vocab(cfg.seed, 32000, step_end_frac=0.01)
     table = B.step_end_table_from_vocab(vocab)
     ends = np.flatnonzero(table.numpy())
+    n_direct = ALG1_ITERATIONS_ONE_LAYER if phys_layers == 1 else ALG1_ITERATIONS
     toks = np.stack([W.token_ids(cfg.seed, T, len(vocab), ends, cfg.boundary_density, sub=500 + i)
-                     for i in range(ALG1_ITERATIONS + 2 + ALG1_GRAPH_ITERATIONS + 2)])
+                     for i in range(n_direct + 2 + ALG1_GRAPH_ITERATIONS + 2)])
     toks[toks == 0] = 1                                            # id 0 is the end-of-sequence token here: nobody completes
     table_d, toks_d = table.to(dev), torch.from_numpy(toks).to(dev)
     q = torch.stack([s["q"][:phys_layers] for s in sets]).contiguous()
@@ -635,14 +640,14 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     run(toks_d[:2], 2)                                              # warm-up
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    r = run(toks_d[2:2 + ALG1_ITERATIONS], ALG1_ITERATIONS)
+    r = run(toks_d[2:2 + n_direct], n_direct)
     e1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / ALG1_ITERATIONS
+    ms = e0.elapsed_time(e1) / n_direct
     # the same loop with each ring slot's iteration recorded as a CUDA graph (on a stream that can be captured); the
     # timed call records its two graphs itself, so that cost is inside the figure
     n_g = ALG1_GRAPH_ITERATIONS if phys_layers == 1 else 6
-    base = 2 + ALG1_ITERATIONS
+    base = 2 + n_direct
     side = torch.cuda.Stream(device=dev)
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
@@ -678,7 +683,7 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     code, bits = pool.last_error()
     return {"iterations": r["iterations"], "ms_per_iteration": ms, "trace_decode_steps_per_s": T / (ms * 1e-3),
             "vs_python_driven_step": None if ms_per_step_python is None else ms_per_step_python / ms,
-            "layers_per_iteration": phys_layers, "launches_per_iteration": 8 + phys_layers,
+            "layers_per_iteration": phys_layers, "launches_per_iteration": 4 + phys_layers,
             "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
             "recorded_iterations": {"iterations": rg["iterations"], "ms_per_iteration": ms_g,
                                     "trace_decode_steps_per_s": T / (ms_g * 1e-3), "vs_direct_launches": ms / ms_g,
@@ -730,6 +735,21 @@ def scorer_measurements(cfg, dev, rows=65536, reps=20, all_rows_density=1.0):
         res[name] = {"rows": M, "boundary_rows": nbr, "us_per_call": ms * 1e3, "rows_per_s": nbr / (ms * 1e-3),
                      "tflops": tfl, "frac_of_bf16_peak": tfl / peak,
                      "first_layer": ("tcgen05, %d units per CTA" % info["tc_units"]) if info["tc_units"] else "cuda cores"}
+        if name == "decode":
+            # a call this short is bound by the host's launch rate when timed back to back: queue the calls behind a
+            # kernel that keeps the GPU busy, so that the events see the device's own time; and once more with the L2
+            # flushed before every call (in a decode step the attention launches have just streamed gigabytes through it)
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+            for cold in (False, True):
+                ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+                torch.cuda._sleep(int(2e7))
+                for a_, b_ in ev:
+                    if cold:
+                        flush.zero_()
+                    a_.record(); pool.score_steps(hid[:M], mask, rt[:M], wts, out[:M]); b_.record()
+                torch.cuda.synchronize()
+                res[name]["us_per_call_device" + ("_cold_l2" if cold else "")] = float(np.median([a_.elapsed_time(b_) for a_, b_ in ev])) * 1e3
+            del flush
     code, mask_bits = pool.last_error()
     res["device_error_mask"] = mask_bits
     pool.close()

@@ -10,7 +10,8 @@
 // outputs: the caller supplies, per iteration, the sampled token of every trace, the new K/V rows, the
 // queries of every layer and the last-layer hidden states; this file chains the library's own steps on
 // them - cache write, attention over the paged cache, step-end detection, scorer, completion of traces
-// that sampled the end-of-sequence token, memory trigger and eviction - without a host round trip: row i
+// that sampled the end-of-sequence token, memory trigger and eviction (four launches besides the attention's) -
+// without a host round trip: row i
 // of every input is trace i, and traces that are no longer live are passed over on the device.
 // One trigger check is made per iteration (a batch of NextToken calls), after the batch's cache writes.
 //
@@ -26,36 +27,15 @@ using namespace stepk;
 
 namespace {
 
-// Live traces (ascending) -> it_ids, those whose sampled token is the end-of-sequence token -> it_fin.
-__global__ void __launch_bounds__(1024)
-iter_prepare_kernel(DevViews v, Geo g, int n, const int32_t* __restrict__ token_ids, int eos_token) {
-  __shared__ int s_warp[33];
-  int n_live = 0, n_fin = 0;
-  for (int base = 0; base < n; base += blockDim.x) {
-    const int t = base + threadIdx.x;
-    const int lv = t < n && v.live[t];
-    const int fin = lv && token_ids[t] == eos_token;
-    int total;
-    int at = block_excl_scan(lv, s_warp, &total);
-    if (lv) v.it_ids[n_live + at] = t;
-    n_live += total;
-    at = block_excl_scan(fin, s_warp, &total);
-    if (fin) v.it_fin[n_fin + at] = t;
-    n_fin += total;
-  }
-  if (threadIdx.x == 0) { v.counters[C_IT_NLIVE] = n_live; v.counters[C_IT_NFIN] = n_fin; }
-}
-
 // Completion: every valid, live listed trace records (score_t, answer) for the vote, then the cluster
 // releases their KV exactly as an eviction would.  n_dev (may be null) caps the list on the device;
 // answers are indexed by trace id (by_trace) or by position in the list.
-__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kPruneThreads, 1)
-finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, const int32_t* __restrict__ n_dev,
-              const int32_t* __restrict__ answers, int by_trace, float unscored) {
+__device__ inline void finish_listed_cluster(DevViews& v, const Geo& g, const int32_t* __restrict__ ids, int n,
+                                             const int32_t* __restrict__ n_dev, const int32_t* __restrict__ answers,
+                                             int by_trace, float unscored, int* s_warp) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  __shared__ int s_warp[33];
-  if (n_dev && *n_dev <= 0) return;      // nobody completes (every CTA reads the same count: the whole cluster leaves)
+  if (n_dev && *n_dev <= 0) return;      // nobody completes (every CTA reads the same count: the whole cluster passes)
   if (cluster.block_rank() == 0) {
     const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
     // an id listed twice completes once, at its first place in the list (v.prune_rank records that place)
@@ -93,6 +73,25 @@ finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, const i
   }
   cluster.sync();
   release_listed_cluster(v, g, __ldcg(&v.counters[C_PRUNE_N]), unscored, s_warp);
+}
+
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kPruneThreads, 1)
+finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, const int32_t* __restrict__ n_dev,
+              const int32_t* __restrict__ answers, int by_trace, float unscored) {
+  __shared__ int s_warp[33];
+  finish_listed_cluster(v, g, ids, n, n_dev, answers, by_trace, unscored, s_warp);
+}
+
+// The end of one iteration of the loop in a single launch: the live traces that sampled the end-of-sequence token
+// complete (v.it_fin, listed by the iteration's cache-write kernel), then the memory trigger is tested and the
+// eviction rule applied up to `tests` times, each test seeing the pool the one before it left.
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kPruneThreads, 1)
+iter_tail_kernel(DevViews v, Geo g, int n, const int32_t* __restrict__ answers, float threshold, float keep_frac, int tests,
+                 float unscored, int32_t* __restrict__ pruned_ids_out, int32_t* __restrict__ n_pruned_out) {
+  __shared__ int s_warp[33];
+  finish_listed_cluster(v, g, v.it_fin, n, v.counters + C_IT_NFIN, answers, 1, unscored, s_warp);
+  for (int k = 0; k < tests; ++k)
+    if (!trigger_and_evict_cluster(v, g, nullptr, threshold, keep_frac, unscored, pruned_ids_out, n_pruned_out, s_warp)) break;
 }
 
 // WeightedVote: total[a] = sum of final scores of the completed traces that answered a; the largest total
@@ -177,31 +176,24 @@ int algorithm1_iteration(step_pool* pool, const step_iteration* it, void* stream
   Geo g = geo_of(pool);
   DevViews& v = pool->v;
   int st;
-  // who is live, who completes
-  iter_prepare_kernel<<<1, 1024, 0, s>>>(v, g, n, it->token_ids, it->eos_token);
-  // NextToken's cache write for the live traces (row t of k_new / v_new belongs to trace t)
-  st = append_kv_impl(pool, v.it_ids, n, 1, it->k_new, it->v_new, v.counters + C_IT_NLIVE, 1, s);
+  // NextToken's cache write for the live traces (row t of k_new / v_new belongs to trace t); the same kernel lists
+  // who is live and who completes
+  st = append_kv_impl(pool, nullptr, n, 1, it->k_new, it->v_new, nullptr, 1, s, it->token_ids, it->eos_token);
   if (st != STEP_OK) return st;
   // NextToken's attention, layer by layer (traces that are not live have length 0 and get zeros)
   st = decode_attention_layers(pool, 0, it->n_layers_attention, it->q, v.block_table, v.seq_lens, n, it->attn_out, stream);
   if (st != STEP_OK) return st;
   // `if x ends a step: y <- f(h); update score_t`
   FlagSource src{nullptr, it->token_ids, it->step_end_table, it->vocab, it->boundary_mask_out, v.live};
-  st = score_steps_impl(pool, it->hidden, src, nullptr, n, it->scorer, it->step_scores_out, stream);
+  st = score_steps_impl(pool, it->hidden, src, nullptr, n, it->scorer, it->step_scores_out, it->trace_scores_out, n, stream);
   if (st != STEP_OK) return st;
-  if (it->trace_scores_out)
-    STEP_CUDA_OK(cudaMemcpyAsync(it->trace_scores_out, v.trace_scores, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, s));
-  // traces that sampled the end-of-sequence token complete
-  finish_kernel<<<kClusterCtas, kPruneThreads, 0, s>>>(v, g, v.it_fin, n, v.counters + C_IT_NFIN, it->answers, 1,
-                                                       pool->cfg.unscored_score);
-  // `if GPUMemoryFull: evict`
+  // traces that sampled the end-of-sequence token complete; `if GPUMemoryFull: evict`
   int32_t* pruned = it->pruned_ids_out ? it->pruned_ids_out : v.it_pruned;
   int32_t* n_pruned = it->n_pruned_out ? it->n_pruned_out : v.counters + C_IT_NPRUNED;
   const int tests = it->max_evictions > 1 ? it->max_evictions : 1;
-  for (int k = 0; k < tests; ++k) {
-    st = prune_if_saturated(pool, nullptr, it->threshold, it->keep_frac, pruned, n_pruned, stream);
-    if (st != STEP_OK) return st;
-  }
+  iter_tail_kernel<<<kClusterCtas, kPruneThreads, 0, s>>>(v, g, n, it->answers, it->threshold, it->keep_frac, tests,
+                                                          pool->cfg.unscored_score, pruned, n_pruned);
+  if (launch_ok() != STEP_OK) return STEP_ERR_CUDA;
   return STEP_OK;
 }
 

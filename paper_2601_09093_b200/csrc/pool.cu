@@ -50,6 +50,7 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.score_idx = take(rows * 4);
   l.score_z = take(rows * kScoreSplits * 4);
   l.score_part = take((rows + kScoreFoldRows - 1) / kScoreFoldRows * T * 8);
+  l.score_zs = take((size_t)kSmallRows * kSmallCtas * 4);
   l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
   l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
   l.attn_cnt = take((size_t)kMaxTracesFast * c->num_kv_heads * 4);
@@ -171,10 +172,42 @@ fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __rest
 // ---------------------------------------------------------------- append_kv
 // Phase 1 (one CTA): decide, in list order, which traces get their pages; pop blocks.
 // n_dev (may be null): only the first min(n, *n_dev) listed traces take part; the rest are passed over in silence.
+// ids == nullptr (the loop of Algorithm 1, whose row i is trace i): the list is made here first - the live traces
+// among 0 .. n-1 in ascending order go to v.it_ids, and, if tokens is given, those of them whose sampled token is
+// eos go to v.it_fin (the traces that complete in this iteration); the counts to C_IT_NLIVE / C_IT_NFIN.
 __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, int n_tokens,
-                                    const int32_t* __restrict__ n_dev) {
+                                    const int32_t* __restrict__ n_dev, const int32_t* __restrict__ tokens, int eos) {
   extern __shared__ int sm[];
-  const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
+  dependents_may_launch();                               // the kernel that writes the rows may set itself up meanwhile
+  int n_listed = -1;
+  if (!ids) {
+    __shared__ int s_cnt[2][8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int n_live = 0, n_fin = 0;
+    for (int base = 0; base < n; base += blockDim.x) {
+      const int t = base + threadIdx.x;
+      const bool lv = t < n && v.live[t];
+      const bool fin = lv && tokens && tokens[t] == eos;
+      const unsigned bl = __ballot_sync(0xffffffffu, lv), bf = __ballot_sync(0xffffffffu, fin);
+      __syncthreads();                                   // the counts of the pass before have been read
+      if (lane == 0) { s_cnt[0][warp] = __popc(bl); s_cnt[1][warp] = __popc(bf); }
+      __syncthreads();
+      int bl_before = 0, bf_before = 0, bl_all = 0, bf_all = 0;
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+        if (w < warp) { bl_before += s_cnt[0][w]; bf_before += s_cnt[1][w]; }
+        bl_all += s_cnt[0][w]; bf_all += s_cnt[1][w];
+      }
+      const unsigned below = (1u << lane) - 1;
+      if (lv) v.it_ids[n_live + bl_before + __popc(bl & below)] = t;
+      if (fin) v.it_fin[n_fin + bf_before + __popc(bf & below)] = t;
+      n_live += bl_all; n_fin += bf_all;
+    }
+    if (threadIdx.x == 0) { v.counters[C_IT_NLIVE] = n_live; v.counters[C_IT_NFIN] = n_fin; }
+    __syncthreads();                                     // the list is read back below by other threads
+    ids = v.it_ids;
+    n_listed = n_live;
+  }
+  const int n_eff = n_listed >= 0 ? n_listed : (n_dev ? min(n, max(*n_dev, 0)) : n);
   int* s_need = sm;            // pages wanted, or -1 if the trace is skipped
   int* s_off = sm + n;         // pops that precede this trace's
   int* s_have = sm + 2 * n;
@@ -250,6 +283,7 @@ append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __re
                     const uint4* __restrict__ vnew, const int32_t* __restrict__ ids,
                     int n_tokens, int cpr, int layers_per_cta, int src_by_id) {
   const int idx = blockIdx.x / n_tokens, j = blockIdx.x - idx * n_tokens;
+  wait_for_primary();                                            // launched as a dependent of the allocation kernel
   const int base = v.append_base[idx];
   if (base < 0) return;                                          // this trace's request was not met
   const int t = ids[idx];
@@ -355,6 +389,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.prune_list = (int32_t*)(m + lay.prune_list); v.prune_off = (int32_t*)(m + lay.prune_off);
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
   v.score_part = (float2*)(m + lay.score_part);
+  v.score_zs = (float*)(m + lay.score_zs);
   v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o); v.attn_cnt = (int32_t*)(m + lay.attn_cnt);
   const bool mma = lay.pre_ws_o != lay.pre_ml;      // the regions are zero-sized for other shapes
   v.pre_ws_ml = mma ? (float*)(m + lay.pre_ws_ml) : nullptr; v.pre_ws_o = mma ? (float*)(m + lay.pre_ws_o) : nullptr;
@@ -417,25 +452,29 @@ int kv_pool_fork_prefix(step_pool* pool, int n_traces, int prefix_len, const voi
 
 int append_kv(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
               const void* v_new, void* stream) {
-  return stepk::append_kv_impl(pool, trace_ids, n, n_tokens, k_new, v_new, nullptr, 0, (cudaStream_t)stream);
+  if (!trace_ids && n > 0 && n_tokens > 0) return STEP_ERR_INVALID_ARG;
+  return stepk::append_kv_impl(pool, trace_ids, n, n_tokens, k_new, v_new, nullptr, 0, (cudaStream_t)stream, nullptr, 0);
 }
 
 }  // extern "C"
 
 int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
-                          const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s) {
+                          const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s,
+                          const int32_t* live_tokens, int eos) {
   if (!pool || n < 0 || n_tokens < 0) return STEP_ERR_INVALID_ARG;
   if (n == 0 || n_tokens == 0) return STEP_OK;
-  if (!trace_ids || !k_new || !v_new) return STEP_ERR_INVALID_ARG;
+  if (!k_new || !v_new) return STEP_ERR_INVALID_ARG;
   if (n > pool->cfg.max_traces) return STEP_ERR_INVALID_ARG;   // ids must be distinct
   Geo g = geo_of(pool);
   const int cpe = 16 / pool->elem_bytes, cpr = g.d / cpe;
   const size_t row_chunks = (size_t)n_tokens * g.L * g.Hkv * cpr;   // 16-byte chunks of K (or V) per trace
   constexpr int kListChunk = 2048;                                  // traces per launch (24 KiB of shared memory for the scan)
+  if (!trace_ids && (n > kListChunk || !src_by_id)) return STEP_ERR_INVALID_ARG;   // the live-trace form is one launch, rows by trace id
   for (int off = 0; off < n; off += kListChunk) {
     const int m = n - off < kListChunk ? n - off : kListChunk;
     if (n_dev && off > 0) return STEP_ERR_INVALID_ARG;              // a device-side count covers one launch only
-    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens, n_dev);
+    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids ? trace_ids + off : nullptr, m, n_tokens, n_dev,
+                                                                    live_tokens, eos);
     const size_t src_off = src_by_id ? 0 : row_chunks * off;
     // enough CTAs to occupy the device: (trace, token) pairs x splits of the layer range
     const long long pairs = (long long)m * n_tokens;
@@ -445,9 +484,11 @@ int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int 
     if (splits < 1) splits = 1;
     const int layers_per_cta = (g.L + splits - 1) / splits;
     splits = (g.L + layers_per_cta - 1) / layers_per_cta;
-    append_write_kernel<<<dim3((unsigned)pairs, (unsigned)splits), 256, 0, s>>>(
-        pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off,
-        (const uint4*)v_new + src_off, trace_ids + off, n_tokens, cpr, layers_per_cta, src_by_id);
+    // a programmatic dependent of the allocation kernel: scheduled while that one runs, waits for it before its first read
+    if (launch_dependent(append_write_kernel, dim3((unsigned)pairs, (unsigned)splits), dim3(256), 0, s, pool->v, g,
+                         (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off, (const uint4*)v_new + src_off,
+                         trace_ids ? trace_ids + off : (const int32_t*)pool->v.it_ids, n_tokens, cpr, layers_per_cta, src_by_id) != cudaSuccess)
+      return STEP_ERR_CUDA;
   }
   return launch_ok();
 }

@@ -163,4 +163,79 @@ __device__ inline void release_listed_cluster(DevViews& v, const Geo& g, int n_l
   cluster.sync();                        // no CTA leaves while its count may still be read
 }
 
+// The memory trigger and the eviction (Sec. 3.2; Algorithm 1, the GPUMemoryFull branch) for a cluster of kClusterCtas
+// CTAs: every CTA evaluates the trigger (same inputs, same answer); rank 0 ranks the traces and lists the evicted
+// ones; the cluster releases them together.
+// Called by every CTA of the cluster; true if the trigger fired (the same answer in every CTA).
+__device__ inline bool trigger_and_evict_cluster(DevViews& v, const Geo& g, const float* __restrict__ scores_in, float threshold,
+                                                 float keep_frac, float unscored, int32_t* __restrict__ pruned_ids_out,
+                                                 int32_t* __restrict__ n_pruned_out, int* s_warp) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const bool leader = cluster.block_rank() == 0;
+  __shared__ int s_nlive, s_need, s_go, s_nkeep;
+  const float* scores = scores_in ? scores_in : v.trace_scores;
+  const int T = g.max_traces;
+  if (threadIdx.x == 0) { s_nlive = 0; s_need = 0; }
+  __syncthreads();
+  // ---- 1. the trigger
+  int nl = 0, nd = 0;
+  for (int t = threadIdx.x; t < T; t += blockDim.x)
+    if (v.live[t]) { ++nl; nd += (v.seq_lens[t] % g.P) == 0; }
+  if (nl) atomicAdd(&s_nlive, nl);
+  if (nd) atomicAdd(&s_need, nd);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int used = g.num_blocks - v.counters[C_FREE_COUNT];
+    const long long limit = (long long)floor((double)threshold * (double)g.num_blocks);
+    int go = (long long)used + s_need > limit;
+    int n_keep = 0;
+    if (go) {
+      n_keep = keep_frac < 0.f ? s_nlive - 1 : (int)ceil((double)keep_frac * (double)s_nlive - 1e-6);
+      if (keep_frac >= 0.f && n_keep < 1) n_keep = 1;
+      if (s_nlive == 0 || n_keep >= s_nlive) go = 0;
+    }
+    s_go = go; s_nkeep = n_keep;
+    if (!go && leader) *n_pruned_out = 0;
+  }
+  __syncthreads();
+  if (!s_go) return false;                // the whole cluster leaves: nothing has been written yet
+  const int n_keep = s_nkeep;
+  if (leader) {
+    // ---- 2. rank by counting: a warp per trace, lanes over rivals
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int t = warp; t < T; t += nwarps) {
+      int evict = 0;
+      if (v.live[t]) {
+        const float st = scores[t];
+        int ahead = 0;
+        for (int u = lane; u < T; u += 32)
+          if (u != t && v.live[u] && orders_before(scores[u], u, st, t)) ++ahead;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
+        evict = ahead >= n_keep;
+      }
+      if (lane == 0) v.prune_rank[t] = evict;
+    }
+    __syncthreads();
+    // ---- 3. evicted ids, ascending
+    int n_list = 0;
+    for (int base = 0; base < T; base += blockDim.x) {
+      const int t = base + threadIdx.x;
+      const int f = t < T ? v.prune_rank[t] : 0;
+      int chunk_total;
+      const int at = block_excl_scan(f, s_warp, &chunk_total);
+      if (f) { v.prune_list[n_list + at] = t; pruned_ids_out[n_list + at] = t; }
+      n_list += chunk_total;
+    }
+    if (threadIdx.x == 0) { *n_pruned_out = n_list; v.counters[C_PRUNE_N] = n_list; v.counters[C_N_EVICTED] += n_list; }
+    __threadfence();
+  }
+  cluster.sync();
+  // ---- 4. release
+  release_listed_cluster(v, g, __ldcg(&v.counters[C_PRUNE_N]), unscored, s_warp);
+  return true;
+}
+
+
 }  // namespace stepk

@@ -15,6 +15,9 @@
 //   finish  : fixed-order sum of the slices, + b2, sigmoid, scatter to the row; then every trace's new
 //             scores are folded into its (sum, count) in ascending row order (per 512-row CTA, the
 //             CTA partials in CTA order) and the mean is refreshed.
+// A call with at most kSmallRows candidate rows - the shape of a decode step, one row per trace - does all of
+// that in ONE launch (score_small_kernel): the three-launch form costs more in launch gaps than such a call
+// has work.
 #include "step_internal.cuh"
 #include "block_scan.cuh"
 
@@ -291,6 +294,217 @@ score_finish_kernel(DevViews v, Geo g, const int32_t* __restrict__ row_trace, in
   }
 }
 
+// ---------------------------------------------------------------- one launch for a decode step's rows
+// grid = S CTAs, CTA c owns hidden units [c * mu, (c + 1) * mu).  Every CTA builds the same ascending list of
+// step-end rows from the flags (M <= kSmallRows, one thread per row; only CTA 0 writes mask_out and error flags),
+// then, for tiles of kRowTile listed rows staged in shared memory as fp32, its warps take the CTA's units one by
+// one (lanes over D, 16-byte loads of the W1 row) and the CTA's partial w2 . ReLU(W1 h + b1) per row goes to
+// score_zs[row][c].  The CTA that finishes last adds the partials in CTA order, applies b2 and the sigmoid, writes
+// every row's output (NaN where no step ends), folds the new scores into the traces' running means in ascending
+// row order and refreshes the means.  Dynamic shared memory: kRowTile * D floats.
+template <typename T> __device__ inline void load4(const T* p, float (&w)[4]);
+template <> __device__ inline void load4<float>(const float* p, float (&w)[4]) {
+  const float4 x = *reinterpret_cast<const float4*>(p);
+  w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+}
+template <> __device__ inline void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&w)[4]) {
+  const uint2 x = *reinterpret_cast<const uint2*>(p);
+  w[0] = __uint_as_float(x.x << 16); w[1] = __uint_as_float(x.x & 0xffff0000u);
+  w[2] = __uint_as_float(x.y << 16); w[3] = __uint_as_float(x.y & 0xffff0000u);
+}
+
+constexpr int kSmallThreads = 256;
+constexpr int kSmallWarps = kSmallThreads / 32;
+
+template <typename T>
+__global__ void __launch_bounds__(kSmallThreads)
+score_small_kernel(DevViews v, Geo g, FlagSource src, const T* __restrict__ hidden, const int32_t* __restrict__ row_trace,
+                   int M, const T* __restrict__ W1, const T* __restrict__ b1, const T* __restrict__ w2, float b2,
+                   int D, int m, float unscored, float* __restrict__ step_scores, float* __restrict__ trace_scores_out, int n_out) {
+  extern __shared__ float s_h[];                      // [kRowTile][D]
+  __shared__ int s_list[kSmallRows];
+  __shared__ int s_wcnt[kSmallWarps + 1];
+  __shared__ float s_part[kSmallWarps][kRowTile];
+  __shared__ float s_y[kSmallRows];
+  __shared__ int s_tr[kSmallRows];
+  __shared__ int s_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = gridDim.x, c = blockIdx.x;
+  const int mu = (m + S - 1) / S;
+  const int j0 = c * mu, j1 = min(m, j0 + mu);
+  const bool vec4 = D % 4 == 0 && ((uintptr_t)W1 & 15) == 0;
+  // The W1 row of this warp's first unit does not depend on which rows end a step: its loads (the first kPrefetch
+  // steps of four elements per lane) are issued before anything else, so that their latency - W1 is usually not in
+  // the L2 - runs alongside the flag scan and the staging of the hidden rows.
+  constexpr int kPrefetch = 32;
+  float wpre[kPrefetch][4];
+  if (vec4 && j0 + warp < j1) {
+    const T* wrow = W1 + (size_t)(j0 + warp) * D;
+#pragma unroll
+    for (int u = 0; u < kPrefetch; ++u)
+      if (lane * 4 + u * 128 < D) load4(wrow + lane * 4 + u * 128, wpre[u]);
+  }
+  // ---- the list of step-end rows (the same in every CTA)
+  FlagSource quiet = src;
+  if (c != 0) quiet.mask_out = nullptr;
+  int32_t* err = c == 0 ? v.counters : nullptr;
+  bool f = false;
+  if ((int)threadIdx.x < M) {
+    if (quiet.live && !quiet.live[threadIdx.x]) { if (quiet.mask_out) quiet.mask_out[threadIdx.x] = 0; }
+    else if (!quiet.tokens) f = quiet.mask[threadIdx.x] != 0;
+    else {
+      const int id = quiet.tokens[threadIdx.x];
+      if (id < 0 || id >= quiet.vocab) { if (err) flag_error(err, STEP_ERR_INVALID_ARG); }
+      else f = quiet.table[id] != 0;
+      if (quiet.mask_out) quiet.mask_out[threadIdx.x] = f ? 1 : 0;
+    }
+  }
+  const unsigned bal = __ballot_sync(0xffffffffu, f);
+  if (lane == 0) s_wcnt[warp] = __popc(bal);
+  __syncthreads();
+  int before = 0, nb = 0;
+  for (int w = 0; w < kSmallWarps; ++w) { if (w < warp) before += s_wcnt[w]; nb += s_wcnt[w]; }
+  if (f) s_list[before + __popc(bal & ((1u << lane) - 1))] = threadIdx.x;
+  __syncthreads();
+  // ---- this CTA's units, tile by tile of the listed rows
+  for (int r0 = 0; r0 < nb && j0 < j1; r0 += kRowTile) {
+    const int rows = min(kRowTile, nb - r0);
+    if (vec4 && ((uintptr_t)hidden & 15) == 0) {
+      // all rows' loads first (four elements per thread and step), then the stores
+      for (int k = threadIdx.x * 4; k < D; k += blockDim.x * 4) {
+        float hv[kRowTile][4];
+#pragma unroll
+        for (int r = 0; r < kRowTile; ++r)
+          if (r < rows) load4(hidden + (size_t)s_list[r0 + r] * D + k, hv[r]);
+#pragma unroll
+        for (int r = 0; r < kRowTile; ++r)
+          *reinterpret_cast<float4*>(&s_h[r * D + k]) = r < rows ? make_float4(hv[r][0], hv[r][1], hv[r][2], hv[r][3])
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    } else {
+      for (int r = 0; r < kRowTile; ++r) {
+        if (r < rows) {
+          const T* hs = hidden + (size_t)s_list[r0 + r] * D;
+          for (int k = threadIdx.x; k < D; k += blockDim.x) s_h[r * D + k] = cvt(hs[k]);
+        } else {
+          for (int k = threadIdx.x; k < D; k += blockDim.x) s_h[r * D + k] = 0.f;
+        }
+      }
+    }
+    __syncthreads();
+    float zpart[kRowTile];
+#pragma unroll
+    for (int r = 0; r < kRowTile; ++r) zpart[r] = 0.f;
+    for (int j = j0 + warp; j < j1; j += kSmallWarps) {
+      const T* wrow = W1 + (size_t)j * D;
+      float acc[kRowTile];
+#pragma unroll
+      for (int r = 0; r < kRowTile; ++r) acc[r] = 0.f;
+      if (vec4) {
+        // four consecutive k per lane and step: one 8- or 16-byte load of the W1 row, one 16-byte load per staged
+        // hidden row.  W1 is usually not in the L2 (the attention launches before this call stream gigabytes through
+        // it), so the loads of eight steps are issued together: what this loop costs is its dependent round trips.
+        int k_from = lane * 4;
+        if (j == j0 + warp) {
+          // this warp's first unit: the prefetched part of its row
+#pragma unroll
+          for (int u = 0; u < kPrefetch; ++u) {
+            if (lane * 4 + u * 128 < D) {
+#pragma unroll
+              for (int r = 0; r < kRowTile; ++r) {
+                const float4 hv = *reinterpret_cast<const float4*>(&s_h[r * D + lane * 4 + u * 128]);
+                acc[r] += wpre[u][0] * hv.x + wpre[u][1] * hv.y + wpre[u][2] * hv.z + wpre[u][3] * hv.w;
+              }
+            }
+          }
+          k_from += kPrefetch * 128;
+        }
+        for (int k0 = k_from; k0 < D; k0 += 128 * 8) {
+          float wv[8][4];
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            if (k0 + u * 128 < D) load4(wrow + k0 + u * 128, wv[u]);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            if (k0 + u * 128 < D) {
+#pragma unroll
+              for (int r = 0; r < kRowTile; ++r) {
+                const float4 hv = *reinterpret_cast<const float4*>(&s_h[r * D + k0 + u * 128]);
+                acc[r] += wv[u][0] * hv.x + wv[u][1] * hv.y + wv[u][2] * hv.z + wv[u][3] * hv.w;
+              }
+            }
+          }
+        }
+      } else {
+        for (int k = lane; k < D; k += 32) {
+          const float wv = cvt(wrow[k]);
+#pragma unroll
+          for (int r = 0; r < kRowTile; ++r) acc[r] += wv * s_h[r * D + k];
+        }
+      }
+      const float bj = cvt(b1[j]), wj = cvt(w2[j]);
+#pragma unroll
+      for (int r = 0; r < kRowTile; ++r) {
+        float x = acc[r];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        zpart[r] += wj * fmaxf(x + bj, 0.f);
+      }
+    }
+    if (lane == 0)
+      for (int r = 0; r < kRowTile; ++r) s_part[warp][r] = zpart[r];
+    __syncthreads();
+    if ((int)threadIdx.x < rows) {
+      float z = 0.f;
+      for (int w = 0; w < kSmallWarps; ++w) z += s_part[w][threadIdx.x];       // warps in order: a fixed sum
+      v.score_zs[(size_t)(r0 + threadIdx.x) * kSmallCtas + c] = z;
+    }
+    __syncthreads();
+  }
+  // ---- whoever finishes last completes the call
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&v.counters[C_SCORE_TICKET], 1) == S - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const int used = min(S, (m + mu - 1) / mu);                                   // CTAs that own units
+  const float nan = __int_as_float(0x7fc00000);
+  if ((int)threadIdx.x < M && !f) step_scores[threadIdx.x] = nan;
+  // a warp per listed row: lane l adds the partials of CTAs l, l + 32, ... in that order, then the lanes are added
+  // in a fixed tree - the same sum whoever is last
+  for (int i = warp; i < nb; i += kSmallWarps) {
+    float z = 0.f;
+    for (int k = lane; k < used; k += 32) z += __ldcg(&v.score_zs[(size_t)i * kSmallCtas + k]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    if (lane == 0) {
+      z += b2;
+      const float y = 1.f / (1.f + expf(-z));
+      const int row = s_list[i];
+      step_scores[row] = y;
+      const int tr = row_trace ? row_trace[row] : row;
+      if (tr < 0 || tr >= g.max_traces) flag_error(v.counters, STEP_ERR_BAD_TRACE);   // names no trace of this pool
+      s_y[i] = y; s_tr[i] = tr;
+    }
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < g.max_traces; t += blockDim.x) {
+    float sum = v.score_sum[t];
+    int cnt = v.score_cnt[t];
+    for (int i = 0; i < nb; ++i)
+      if (s_tr[i] == t) { sum += s_y[i]; ++cnt; }
+    v.score_sum[t] = sum; v.score_cnt[t] = cnt;
+    const float mean = cnt > 0 ? sum / (float)cnt : unscored;
+    v.trace_scores[t] = mean;
+    if (trace_scores_out && t < n_out) trace_scores_out[t] = mean;
+  }
+  if (threadIdx.x == 0) {
+    v.counters[C_SCORE_TICKET] = 0;
+    v.counters[C_SCORE_NB] = nb; v.counters[C_SCORE_TC] = 0; v.counters[C_SCORE_SLICES] = used;
+  }
+}
+
 // step-end detection alone: mask[i] = table[tokens[i]]
 __global__ void __launch_bounds__(256)
 step_end_kernel(FlagSource src, int M, int32_t* counters) {
@@ -306,7 +520,7 @@ extern "C" int score_steps(step_pool* pool, const void* hidden, const uint8_t* b
   if (M == 0) return STEP_OK;
   if (!boundary_mask) return STEP_ERR_INVALID_ARG;
   FlagSource src{boundary_mask, nullptr, nullptr, 0, nullptr, nullptr};
-  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
+  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, nullptr, 0, stream);
 }
 
 extern "C" int score_steps_tokens(step_pool* pool, const void* hidden, const int32_t* token_ids,
@@ -317,7 +531,7 @@ extern "C" int score_steps_tokens(step_pool* pool, const void* hidden, const int
   if (M == 0) return STEP_OK;
   if (!token_ids || !step_end_table || vocab < 1) return STEP_ERR_INVALID_ARG;
   FlagSource src{nullptr, token_ids, step_end_table, vocab, boundary_mask_out, nullptr};
-  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, stream);
+  return score_steps_impl(pool, hidden, src, row_trace, M, w, step_scores_out, nullptr, 0, stream);
 }
 
 extern "C" int detect_step_ends(step_pool* pool, const int32_t* token_ids, int M, const uint8_t* step_end_table,
@@ -353,13 +567,33 @@ extern "C" int step_end_table_from_vocab(const char* const* token_text, const in
 }
 
 int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
-                            const scorer_weights* w, float* step_scores_out, void* stream) {
+                            const scorer_weights* w, float* step_scores_out, float* trace_scores_out, int n_out, void* stream) {
   if (!hidden || !step_scores_out) return STEP_ERR_INVALID_ARG;
   if (!w->W1 || !w->b1 || !w->w2 || w->D < 1 || w->m < 1) return STEP_ERR_INVALID_ARG;
   if (w->dtype != STEP_BF16 && w->dtype != STEP_FP32) return STEP_ERR_INVALID_ARG;
   const size_t smem = (size_t)kRowTile * w->D * sizeof(float);
   cudaStream_t s = (cudaStream_t)stream;
   Geo g = geo_of(pool);
+  // a decode step's shape: everything in one launch (unless the tensor-core kernel was asked for by name)
+  if (M <= kSmallRows && pool->scorer_mode <= 0 && smem <= 200 * 1024) {
+    int S = (w->m + 3) / 4;                                        // about four hidden units per CTA
+    const int cap = pool->num_sms < kSmallCtas ? pool->num_sms : kSmallCtas;
+    if (S > cap) S = cap;
+    if (w->dtype == STEP_BF16) {
+      auto kern = score_small_kernel<__nv_bfloat16>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+      kern<<<S, kSmallThreads, smem, s>>>(pool->v, g, src, (const __nv_bfloat16*)hidden, row_trace, M, (const __nv_bfloat16*)w->W1,
+                                          (const __nv_bfloat16*)w->b1, (const __nv_bfloat16*)w->w2, w->b2, w->D, w->m,
+                                          pool->cfg.unscored_score, step_scores_out, trace_scores_out, n_out);
+    } else {
+      auto kern = score_small_kernel<float>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
+      kern<<<S, kSmallThreads, smem, s>>>(pool->v, g, src, (const float*)hidden, row_trace, M, (const float*)w->W1, (const float*)w->b1,
+                                          (const float*)w->w2, w->b2, w->D, w->m, pool->cfg.unscored_score, step_scores_out,
+                                          trace_scores_out, n_out);
+    }
+    return launch_ok();
+  }
   const size_t eb = w->dtype == STEP_BF16 ? 2 : 4;
   const bool tc = pool->scorer_mode >= 0 && score_tc_supported(w, hidden);
   const int tc_min_rows = !tc ? 0 : (pool->scorer_mode > 0 ? 1 : pool->scorer_tc_min_rows);
@@ -400,6 +634,9 @@ int stepk::score_steps_impl(step_pool* pool, const void* hidden, FlagSource src,
                          pool->v, g, rt, off, w->b2, pool->cfg.unscored_score, step_scores_out + off) != cudaSuccess)
       return STEP_ERR_CUDA;
   }
+  if (trace_scores_out && n_out > 0)
+    STEP_CUDA_OK(cudaMemcpyAsync(trace_scores_out, pool->v.trace_scores, (size_t)(n_out < g.max_traces ? n_out : g.max_traces) * sizeof(float),
+                                 cudaMemcpyDeviceToDevice, s));
   return launch_ok();
 }
 

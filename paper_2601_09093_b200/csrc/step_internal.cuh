@@ -23,6 +23,8 @@ constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream p
 constexpr int kPrefixPartitions = 1184; // partitions of the shared-prefix pass of decode_attention_shared_prefix (148 SMs x 8 warps)
 constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
 constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
+constexpr int kSmallRows = 256;       // candidate rows up to which score_steps is one launch (a decode step's shape)
+constexpr int kSmallCtas = 148;       // CTAs of that launch at most; score_zs holds this many partial sums per listed row
 constexpr int kScoreFoldRows = 512;    // listed rows one CTA of the scorer's finishing kernel folds into per-trace partials
 
 // C_SCORE_TC: 0 = the launch's boundary rows go through the CUDA-core MLP kernel; otherwise the
@@ -41,7 +43,7 @@ struct MetaLayout {
   size_t block_table, seq_lens, live, score_sum, score_cnt, trace_scores;
   size_t refcount, free_list, claim, counters;
   size_t append_base, prune_rank, prune_list, prune_off;
-  size_t score_idx, score_z, score_part;
+  size_t score_idx, score_z, score_part, score_zs;
   size_t attn_ml, attn_o, attn_cnt;
   size_t pre_ws_ml, pre_ws_o, pre_ml, pre_o;   // shared-prefix attention (zero-sized for pools the tensor-core kernel does not cover)
   size_t final_score, answer, finished, it_ids, it_fin, it_pruned, it_tokens, it_scores;
@@ -53,7 +55,7 @@ struct DevViews {
   float* score_sum; int32_t* score_cnt; float* trace_scores;
   int32_t* refcount; int32_t* free_list; int32_t* claim; int32_t* counters;
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
-  int32_t* score_idx; float* score_z; float2* score_part;
+  int32_t* score_idx; float* score_z; float2* score_part; float* score_zs;
   float* attn_ml; float* attn_o; int32_t* attn_cnt;
   float* pre_ws_ml; float* pre_ws_o; float* pre_ml; float* pre_o;   // null when zero-sized
   float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
@@ -142,10 +144,13 @@ inline cudaError_t launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 b
 }
 
 // ---- pieces the Algorithm 1 driver (algorithm1.cu) chains together
-// append_kv with two extras: *n_dev (device, may be null) caps the number of listed traces on the device, and
-// src_by_id makes trace t read row t of k_new / v_new instead of row (position in the list).
+// append_kv with extras: *n_dev (device, may be null) caps the number of listed traces on the device; src_by_id makes
+// trace t read row t of k_new / v_new instead of row (position in the list); trace_ids == nullptr (with src_by_id, one
+// token) appends to every live trace among 0 .. n-1 - the list is made on the device (v.it_ids, C_IT_NLIVE) together
+// with the list of those whose sampled token live_tokens[t] equals eos (v.it_fin, C_IT_NFIN; live_tokens may be null).
 int append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int n_tokens, const void* k_new,
-                   const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s);
+                   const void* v_new, const int32_t* n_dev, int src_by_id, cudaStream_t s,
+                   const int32_t* live_tokens, int eos);
 
 // Where score_steps takes a row's step-end flag from: mask[i], or table[tokens[i]] (a token ends a step if its
 // text contains two newlines in a row; the table records that per vocabulary entry).  live (may be null)
@@ -158,8 +163,9 @@ struct FlagSource {
   uint8_t* mask_out;         // [M], or nullptr
   const uint8_t* live;       // [M], or nullptr
 };
+// trace_scores_out (may be null): its first n_out entries get the trace scores as they stand after this call.
 int score_steps_impl(step_pool* pool, const void* hidden, FlagSource src, const int32_t* row_trace, int M,
-                     const scorer_weights* w, float* step_scores_out, void* stream);
+                     const scorer_weights* w, float* step_scores_out, float* trace_scores_out, int n_out, void* stream);
 
 // ---- tensor-core scorer (scorer_tc.cu)
 // True if the tcgen05 kernel covers this scorer shape and these pointers.
