@@ -488,6 +488,7 @@ def run_ours(args):
         res["algorithm1_loop"] = algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log, ids_host,
                                                         ms_total / K if phys_layers == L else None)
         res["scorer"] = scorer_measurements(cfg, dev, rows=args.scorer_rows)
+        res["append_kv"] = append_measurements(cfg, dev, min(phys_layers, 36))
         if args.workload == "c3":
             # last: this consumes the benchmark state (the pool ends with two live traces)
             cyc = prune_cycles(pool, cfg, nb, T, dev, wts, append_log, phys_layers, peak)
@@ -774,6 +775,42 @@ def scorer_measurements(cfg, dev, rows=65536, reps=20, all_rows_density=1.0):
 
 
 WINDOW = 16                         # whole decode steps timed before each saturation point and after each prune
+
+
+def append_measurements(cfg, dev, layers, reps=20):
+    """append_kv alone on a pool of its own: the decode step's call (one new token for every trace, all `layers`
+    layers), timed on the device with the calls queued behind a kernel that keeps the GPU busy, and a bulk call
+    (32 tokens per trace), whose bytes (read + written) are set against the measured copy peak."""
+    import torch
+    from paper_2601_09093_b200 import harness as H, workloads as W
+    T = cfg.n_traces
+    c = W.scaled(cfg, num_layers=layers)
+    bulk = 32
+    pages = T * (2 + (reps + 8) * bulk // c.page_size + (2 * reps + 40) // c.page_size + 2) + 8
+    pool = H.make_pool(c, pages, pages // T + 2, T, device=dev)
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.seed + 99)
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    ids = torch.tensor(pool.fork_prefix(T, 16, rnd(layers, c.num_kv_heads, 16, c.head_dim), rnd(layers, c.num_kv_heads, 16, c.head_dim)),
+                       dtype=torch.int32, device=dev)
+    k1, v1 = rnd(T, 1, layers, c.num_kv_heads, c.head_dim), rnd(T, 1, layers, c.num_kv_heads, c.head_dim)
+    kb, vb = rnd(T, bulk, layers, c.num_kv_heads, c.head_dim), rnd(T, bulk, layers, c.num_kv_heads, c.head_dim)
+    peak, kind = measured_peaks()
+    res = {"traces": T, "layers": layers}
+    for name, kk, vv, n_tok in (("one_token", k1, v1, 1), ("bulk_32_tokens", kb, vb, bulk)):
+        for _ in range(3):
+            pool.append_kv(ids, n_tok, kk, vv)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        torch.cuda._sleep(int(2e7))
+        for a_, b_ in ev:
+            a_.record(); pool.append_kv(ids, n_tok, kk, vv); b_.record()
+        torch.cuda.synchronize()
+        us = float(np.median([a_.elapsed_time(b_) for a_, b_ in ev])) * 1e3
+        moved = 2 * 2 * kk.numel() * 2                       # K and V, read and written, two bytes each
+        res[name] = {"us_per_call_device": us, "bytes_read_and_written": moved, "gbs": moved / us / 1e3,
+                     "frac_of_copy_peak": moved / us / 1e3 / peak}
+    res["device_error_mask"] = pool.last_error()[1]
+    pool.close()
+    return res
 
 
 def prune_cycles(pool, cfg, nb, T, dev, wts, append_log, phys_layers, hbm_peak, n_cycles=5):

@@ -383,6 +383,13 @@ int kv_pool_read_kv(step_pool* pool, int layer, int kv_head, const int32_t* bloc
 /* Tuning knobs of decode_attention (0 keeps the current value): CTAs per launch, and whether
  * the tensor-core bf16 path may be used (1) or the scalar kernel is forced (-1). */
 int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path);
+/* How long the tensor-core kernel of decode_attention (all its entry points) waits for a page copy before it gives
+ * up: the warp then sets the STEP_ERR_TIMEOUT bit of the status word, waits (with
+ * the full limit) for the copies it still has in flight, and leaves; outputs of such a launch are undefined and the
+ * tickets of its split sequences may be left mid-count, so call kv_pool_reset (or destroy the pool) before the next
+ * decode_attention (decode_attention_static clears its own tickets on every call).  Default 2,000,000,000 ns.  0 = no waiting at all: a page that has not landed by the time it
+ * is first looked at counts as timed out - for testing this path, which no healthy device otherwise reaches. */
+int kv_pool_set_wait_limit_ns(step_pool* pool, unsigned long long ns);
 /* Which first-layer kernel score_steps uses for bf16 scorers whose shape the tensor-core kernel covers
  * (D a multiple of 64, m a multiple of 64 and <= 1024, 16-byte aligned W1 and hidden): mode 0 (default)
  * sends a launch to the tensor cores when it has at least tc_min_rows boundary rows (the count is taken

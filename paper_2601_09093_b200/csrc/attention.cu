@@ -135,6 +135,7 @@ struct AttnArgs {
   int pp;                          // shared pages
   int tpb, n_bundles;              // prefix pass: traces per 16-row bundle of query rows, number of bundles
   int q_from_primary;              // 1: the launch before this one in the stream writes q (see decode_attention_dependent)
+  unsigned long long wait_ns;      // limit of the wait for a page copy (the waits that drain copies after a time-out keep the full limit)
 };
 
 // kMode of attn_mma_kernel: the plain kernel; the pass over the shared pages, whose 16 query rows are the G heads of
@@ -317,6 +318,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   int stage = 0;
   uint32_t parity = 0;
   bool alive = true;
+  int timed_out_at = 0;
 
   // ldmatrix lane addressing inside a page (swizzled 16-byte chunks: chunk' = chunk ^ (row & 7))
   const int mi = lane >> 3, r8 = lane & 7;
@@ -359,9 +361,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
       seg_open = true;
     }
 
-    if (!mbar_wait_bounded(my_bar_u32 + stage * 8, parity)) {
+    if (!mbar_wait_bounded(my_bar_u32 + stage * 8, parity, a.wait_ns)) {
       if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
       alive = false;
+      timed_out_at = i;
       break;
     }
     const uint32_t kpage = my_pages_u32 + stage * kPageBytes;
@@ -605,12 +608,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   before_first_write();
   fill_empty_traces();
   if (!alive) {
-    // A wait ran out.  Copies already issued still target this CTA's shared memory, so give each
-    // of them one more bounded wait before the warp leaves; nothing else is touched.
-    for (int s = 0; s < kStages; ++s) {
-      mbar_wait_bounded(my_bar_u32 + s * 8, 0);
-      mbar_wait_bounded(my_bar_u32 + s * 8, 1);
-    }
+    // A wait ran out.  The copies of pages timed_out_at .. issued - 1 were issued and still target this CTA's shared
+    // memory: each gets one more wait, with the full limit, before the warp leaves (page j uses stage j % kStages in
+    // the phase of parity (j / kStages) & 1); nothing else is touched.
+    for (int j = timed_out_at; j < issued; ++j)
+      mbar_wait_bounded(my_bar_u32 + (j % kStages) * 8, (uint32_t)((j / kStages) & 1));
   }
 }
 
@@ -650,6 +652,7 @@ void fill_args(AttnArgs& a, const step_pool* pool, const Geo& g, int layer, cons
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
   a.prefix_blocks = nullptr; a.pre_ml = nullptr; a.pre_o = nullptr; a.pp = 0; a.tpb = 1; a.n_bundles = 0;
   a.q_from_primary = 0;
+  a.wait_ns = pool->wait_limit_ns;
 }
 
 bool mma_shape(const step_pool* pool, const Geo& g, int n) {

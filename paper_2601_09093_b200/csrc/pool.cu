@@ -373,6 +373,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->num_sms = sms;
   p->attn_grid = sms;
   p->fast_path = 1;
+  p->wait_limit_ns = 2000000000ull;
   p->scorer_mode = 0;
   p->scorer_tc_min_rows = 1;
   p->tmap_w1 = nullptr; p->tmap_D = 0; p->tmap_m = 0; p->tc_smem_set = false;
@@ -559,6 +560,12 @@ int kv_pool_read_kv(step_pool* pool, int layer, int kv_head, const int32_t* bloc
       g, (const uint4*)pool->cfg.kv_storage, layer, kv_head, block_row, seq_len, (uint4*)k_out, (uint4*)v_out,
       cpr, cpe, pool->v.counters);
   return launch_ok();
+}
+
+int kv_pool_set_wait_limit_ns(step_pool* pool, unsigned long long ns) {
+  if (!pool) return STEP_ERR_INVALID_ARG;
+  pool->wait_limit_ns = ns;
+  return STEP_OK;
 }
 
 int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path) {

@@ -74,6 +74,7 @@ struct step_pool {
   int num_sms;
   int attn_grid;      // CTAs of the tensor-core attention launch
   int fast_path;      // 1 allowed, -1 forced off
+  unsigned long long wait_limit_ns;   // limit of decode_attention's wait for a page copy (kv_pool_set_wait_limit_ns)
   int scorer_mode;    // 0: tensor-core MLP for launches with >= scorer_tc_min_rows boundary rows; 1: always; -1: never
   int scorer_tc_min_rows;
   // the tensor map of the last W1 the tensor-core scorer was given (encoding it costs a few host microseconds)
