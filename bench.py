@@ -447,7 +447,7 @@ def run_ours(args):
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
                      "traffic": None if traffic_ratio is None else algo_bytes * traffic_ratio,
                      "traffic_source": traffic_src,
-                     "kernel": "decode_attention_layers (attn_mma_kernel, split partials merged in the same launch), per layer",
+                     "kernel": "decode_attention_layers (attn_mma_kernel plus attn_merge_kernel, which combines the split partials), per layer",
                      "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": attn_avg_ms,
                      "min_launch_ms": float(np.min(attn_ms)), "launches_timed": attn_launches,
                      "how_timed": "CUDA events around each decode_attention_layers call (all layers of a step: every launch after "
@@ -476,7 +476,7 @@ def run_ours(args):
         # the same launches counted the way a per-trace kernel would see them (the shared prompt once per trace)
         "kv_gbs_logical": float(np.sum(seq_now - K // 2)) * cfg.bytes_per_token_layer / (attn_avg_ms * 1e-3) / 1e9,
         "attention_share_of_step": float(np.sum(attn_run_ms)) / ms_total,
-        "gpu_launches": K * (2 + L + 1 + 1), "clocks": clocks,
+        "gpu_launches": K * (2 + 2 * L + 1 + 1), "clocks": clocks,
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
     if e2e:

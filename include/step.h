@@ -383,6 +383,13 @@ int kv_pool_read_kv(step_pool* pool, int layer, int kv_head, const int32_t* bloc
 /* Tuning knobs of decode_attention (0 keeps the current value): CTAs per launch, and whether
  * the tensor-core bf16 path may be used (1) or the scalar kernel is forced (-1). */
 int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path);
+/* How decode_attention's tensor-core launch spreads the KV pages over the SMs.  Of every (trace, KV head)
+ * sequence the last dynamic_sixteenths / 16 of its pages (0 .. 12; default 4) are cut into chunks of at least
+ * min_chunk_pages pages (0 keeps the current value; default 16) that warps fetch from a device counter when they
+ * have finished their equal share of the other pages; 0 sixteenths = equal shares only.  The outputs are the same
+ * bits whichever warp processes which chunk.  decode_attention_static and the shared pages' pass of
+ * decode_attention_shared_prefix always use equal shares.  STEP_ERR_INVALID_ARG outside the ranges. */
+int kv_pool_set_attention_balance(step_pool* pool, int dynamic_sixteenths, int min_chunk_pages);
 /* How long the tensor-core kernel of decode_attention (all its entry points) waits for a page copy before it gives
  * up: the warp then sets the STEP_ERR_TIMEOUT bit of the status word, waits (with
  * the full limit) for the copies it still has in flight, and leaves; outputs of such a launch are undefined and the

@@ -109,6 +109,7 @@ def lib():
     L.kv_pool_last_error.argtypes = [vp, C.POINTER(C.c_uint), vp]
     L.kv_pool_read_kv.argtypes = [vp, i, i, vp, i, vp, vp, vp]
     L.kv_pool_set_attention_config.argtypes = [vp, i, i]
+    L.kv_pool_set_attention_balance.argtypes = [vp, i, i]
     L.kv_pool_set_wait_limit_ns.argtypes = [vp, C.c_ulonglong]
     L.scorer_train_workspace_bytes.argtypes = [i, i, i]
     L.scorer_train_workspace_bytes.restype = C.c_size_t
@@ -382,6 +383,10 @@ class KVPool:
 
     def set_attention_config(self, grid_ctas=0, fast_path=0):
         _check("kv_pool_set_attention_config", lib().kv_pool_set_attention_config(self.handle, grid_ctas, fast_path))
+
+    def set_attention_balance(self, dynamic_sixteenths, min_chunk_pages=0):
+        _check("kv_pool_set_attention_balance",
+               lib().kv_pool_set_attention_balance(self.handle, dynamic_sixteenths, min_chunk_pages))
 
     def set_wait_limit_ns(self, ns):
         _check("kv_pool_set_wait_limit_ns", lib().kv_pool_set_wait_limit_ns(self.handle, ns))

@@ -124,7 +124,6 @@ struct AttnArgs {
   float* out;
   float* ws_ml;                    // [partition][2][G][2]
   float* ws_o;                     // [partition][2][G][kD]
-  int32_t* seg_cnt;                // [n][Hkv] tickets of the split sequences; zero between launches
   int32_t* counters;
   int n, Hq, Hkv, G, max_pages, num_blocks;
   float scale_log2;
@@ -135,7 +134,11 @@ struct AttnArgs {
   int pp;                          // shared pages
   int tpb, n_bundles;              // prefix pass: traces per 16-row bundle of query rows, number of bundles
   int q_from_primary;              // 1: the launch before this one in the stream writes q (see decode_attention_dependent)
-  unsigned long long wait_ns;      // limit of the wait for a page copy (the waits that drain copies after a time-out keep the full limit)
+  int32_t* sched;                  // [1] hand-out counter of the chunks, zero between launches; null: equal shares only
+  int dyn16, dyn_chunk;            // sixteenths of every sequence handed out as chunks; smallest chunk (pages)
+  int n_static;                    // equal shares of the static stream: warps of the attention launch
+  int merge_ctas;                  // CTAs of the launch that combines the pieces, at most (one per SM)
+  unsigned long long wait_ns;      // limit of the wait for one page copy
 };
 
 // kMode of attn_mma_kernel: the plain kernel; the pass over the shared pages, whose 16 query rows are the G heads of
@@ -187,51 +190,126 @@ __device__ inline void cursor_next(Cursor& c, const int* cum, int n, int Hkv) {
   c.np = c.t < n ? cum[c.t + 1] - cum[c.t] : 1;
 }
 
+constexpr int kDynSlotBase = 2 * kMaxPartitions;       // partial slots of the chunks follow those of the equal shares
+
+// Largest t with Hkv * cum[t] <= pos (cum is an exclusive prefix sum over the launch's sequences).
+__device__ inline int seek_trace(const int* cum, int n, int Hkv, long long pos) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// ---- the partition of a launch, as both the attention kernel and the kernel that combines the pieces derive it
+// from the launch's lengths.
+// Pages of sequence t of the KV stream (kMode as for attn_mma_kernel); `flag` records what is wrong with a length.
+template <int kMode>
+__device__ inline int seq_pages(const AttnArgs& a, int t, bool flag) {
+  if constexpr (kMode == kPrefixPass) {
+    // a bundle is read if one of its traces holds the whole prefix
+    int pages = 0;
+    for (int u = t * a.tpb; u < (t + 1) * a.tpb && u < a.n; ++u)
+      if (a.seq_lens[u] >= a.pp * kP) pages = a.pp;
+    return pages;
+  } else {
+    int S = a.seq_lens[t];
+    if (S < 0) S = 0;
+    int pages = (S + kP - 1) / kP;
+    if (pages > a.max_pages) { pages = a.max_pages; if (flag) flag_error(a.counters, STEP_ERR_CAPACITY); }
+    if constexpr (kMode == kSuffixPass) {
+      // own pages only; a trace shorter than the prefix it is said to share is flagged and gets zeros
+      if (S >= a.pp * kP) pages -= a.pp;
+      else { pages = 0; if (flag && S > 0) flag_error(a.counters, STEP_ERR_INVALID_ARG); }
+    }
+    return pages;
+  }
+}
+// Pages of sequence t that may go into chunks (before it is known whether the launch has chunks at all).
+__device__ inline int tail_pages(const AttnArgs& a, int pages) { return pages * a.dyn16 / 16; }
+// Pages per chunk, from the sum of tail_pages over the launch's sequences (per KV head); 0: the launch has no chunks.
+// The smallest allowed size, or larger if the chunks would outnumber their partial slots (every sequence's last
+// chunk may be short, hence the 2 * sequences); launches with very many sequences do without the hand-out.
+__device__ inline int chunk_pages(const AttnArgs& a, int n_seq, long long tails) {
+  const long long seqs = (long long)a.Hkv * n_seq;
+  if (!a.sched || a.dyn16 <= 0 || 4 * seqs > kMaxDynChunks) return 0;
+  const long long by_cap = ((long long)a.Hkv * tails + (kMaxDynChunks - 2 * seqs) - 1) / (kMaxDynChunks - 2 * seqs);
+  return (int)(by_cap > a.dyn_chunk ? by_cap : a.dyn_chunk);
+}
+// A sequence of `pages` pages: pa pages in the static stream, ch chunk numbers.  A sequence with a tail has one
+// number per chunk and one more that stands for no pages - its partial slot takes the sequence's static part when
+// that part lies inside a single share.
+__device__ inline void split_seq(const AttnArgs& a, int pages, int C, int& pa, int& ch) {
+  const int tail = C ? tail_pages(a, pages) : 0;
+  pa = pages - tail;
+  ch = tail > 0 ? (tail + C - 1) / C + 1 : 0;
+}
+
+// The whole partition, by one warp, into shared memory: np[n] pages of every sequence, cum[n + 1] its pages in the
+// static stream (prefix sum), cumc[n + 1] its chunk numbers per KV head (prefix sum), *chunk the pages per chunk.
+template <int kMode>
+__device__ inline void build_partition(const AttnArgs& a, int n, int lane, bool flag, int* np, int* cum, int* cumc, int* chunk) {
+  long long tails = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int t = base + lane;
+    if (t < n) {
+      const int pages = seq_pages<kMode>(a, t, flag);
+      np[t] = pages;
+      tails += tail_pages(a, pages);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tails += __shfl_xor_sync(0xffffffffu, tails, o);
+  const int C = chunk_pages(a, n, tails);
+  int run_a = 0, run_c = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int t = base + lane;
+    int pa = 0, ch = 0;
+    if (t < n) split_seq(a, np[t], C, pa, ch);
+    int ia = pa, ic = ch;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int va = __shfl_up_sync(0xffffffffu, ia, o), vc = __shfl_up_sync(0xffffffffu, ic, o);
+      if (lane >= o) { ia += va; ic += vc; }
+    }
+    if (t < n) { cum[t] = run_a + ia - pa; cumc[t] = run_c + ic - ch; }
+    run_a += __shfl_sync(0xffffffffu, ia, 31);
+    run_c += __shfl_sync(0xffffffffu, ic, 31);
+  }
+  if (lane == 0) { cum[n] = run_a; cumc[n] = run_c; *chunk = C; }
+}
+
+// How a launch's pages are spread over the SMs.
+//
+// Every (trace, KV head) sequence is cut in two: its first pages - all but dyn16 sixteenths - belong to the "static"
+// stream (for every trace in order, for every KV head in order, those pages in order), which is cut into one equal
+// contiguous share per warp; its last pages, the "tail", are cut into chunks of C pages, and the chunks of all
+// sequences are handed out at run time, by an atomic counter, to whichever warp has finished what it had.  SMs do
+// not all stream at the same rate (measured: up to 20 % apart), and with equal shares alone a launch lasts as long
+// as its slowest SM while the others idle; the chunks even that out.
+// Which warp processes a chunk is decided at run time, but the pieces themselves - and with them every partial
+// result and the order in which partials are combined - are fixed by the launch's lengths alone, so the outputs do
+// not depend on the hand-out.  This kernel only leaves the partial (max, sum, weighted values) of every piece in
+// the piece's slot; a second launch (attn_merge_kernel, a programmatic dependent of this one) combines the pieces
+// of every sequence.  (An earlier form combined them in this kernel, by tickets: the fence and the atomic round trip
+// at the end of every chunk cost more, in a saturated memory system, than the hand-out gained.)
 template <int kWarps, int kStages, bool kRows16, int kMode>
 __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   static_assert(kMode != kPrefixPass || kRows16, "the prefix pass uses all 16 rows of the tile");
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* s_pages = smem;                                              // [kWarps][kStages][8 KiB]
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kWarps * kStages * kPageBytes);
-  int* s_cum = reinterpret_cast<int*>(s_bar + kWarps * kStages);              // [n + 1]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // n = sequences of the KV stream: traces, or (prefix pass) bundles of tpb traces that share the prefix pages
   const int n = kMode == kPrefixPass ? a.n_bundles : a.n, Hkv = a.Hkv, G = a.G;
+  int* s_np = reinterpret_cast<int*>(s_bar + kWarps * kStages);               // [n]     pages of sequence t
+  int* s_cum = s_np + n;                                                      // [n + 1] its pages in the static stream, prefix sum
+  int* s_cumc = s_cum + n + 1;                                                // [n + 1] chunk numbers of its tail (per KV head), prefix sum
+  int* s_chunk = s_cumc + n + 1;                                              // [1]     pages per chunk (0: no chunks)
 
-  // ---- pages per sequence, exclusive prefix sum (warp 0), barrier init (lane 0 of each warp)
-  if (warp == 0) {
-    int running = 0;
-    for (int base = 0; base < n; base += 32) {
-      const int t = base + lane;
-      int pages = 0;
-      if (t < n) {
-        if constexpr (kMode == kPrefixPass) {
-          // a bundle is read if one of its traces holds the whole prefix
-          for (int u = t * a.tpb; u < (t + 1) * a.tpb && u < a.n; ++u)
-            if (a.seq_lens[u] >= a.pp * kP) pages = a.pp;
-        } else {
-          int S = a.seq_lens[t];
-          if (S < 0) S = 0;
-          pages = (S + kP - 1) / kP;
-          if (pages > a.max_pages) { pages = a.max_pages; flag_error(a.counters, STEP_ERR_CAPACITY); }
-          if constexpr (kMode == kSuffixPass) {
-            // own pages only; a trace shorter than the prefix it is said to share is flagged and gets zeros
-            if (S >= a.pp * kP) pages -= a.pp;
-            else { pages = 0; if (S > 0) flag_error(a.counters, STEP_ERR_INVALID_ARG); }
-          }
-        }
-      }
-      int incl = pages;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (t < n) s_cum[t] = running + incl - pages;
-      running += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) s_cum[n] = running;
-  }
+  // ---- pages per sequence, the chunk size, prefix sums (warp 0), barrier init (lane 0 of each warp)
+  if (warp == 0) build_partition<kMode>(a, n, lane, true, s_np, s_cum, s_cumc, s_chunk);
   if (lane == 0) {
     for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&s_bar[warp * kStages + s]), 1);
     mbar_init_fence();
@@ -240,11 +318,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
   // Nothing has been written yet, and nothing read so far is written by another launch of this kernel: when this
   // launch was scheduled ahead of the completion of such a launch before it (a layer-by-layer sequence of calls made
-  // by the library itself), it may run up to its first write - of an output, a partial or a ticket - and must then
-  // wait for that launch, whose partials and tickets share the scratch.  A no-op for a launch made the plain way.
-  // When the launch before this one is the caller's own kernel that produces q (q_from_primary), the wait moves up to
-  // the first read of q: what precedes it - the prefix sums above, the barriers, and every warp's first kStages page
-  // copies - depends only on the lengths, the block table and the cache, and overlaps that kernel's tail.
+  // by the library itself), it may run up to its first write - of an output, a partial, a ticket or a claim on the
+  // chunk counter - and must then wait for that launch, whose scratch it shares.  A no-op for a launch made the
+  // plain way.  When the launch before this one is the caller's own kernel that produces q (q_from_primary), the
+  // wait moves up to the first read of q: what precedes it - the prefix sums above, the barriers, and every warp's
+  // first kStages page copies - depends only on the lengths, the block table and the cache, and overlaps that
+  // kernel's tail.
   dependents_may_launch();
   bool waited = false;
   auto before_first_write = [&]() { if (!waited) { wait_for_primary(); waited = true; } };
@@ -253,7 +332,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   auto fill_empty_traces = [&]() {
     if constexpr (kMode != kPrefixPass) {
       for (int t = blockIdx.x; t < n; t += gridDim.x)
-        if (s_cum[t + 1] == s_cum[t]) {
+        if (s_np[t] == 0) {
           const bool prefix_only = kMode == kSuffixPass && a.seq_lens[t] >= a.pp * kP;
           for (int k = threadIdx.x; k < a.Hq * kD; k += blockDim.x) {
             float v = 0.f;
@@ -264,28 +343,64 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     }
   };
 
-  const long long total = (long long)Hkv * s_cum[n];
-  const int n_part = gridDim.x * kWarps;
-  const long long W = (total + n_part - 1) / n_part;
+  const int C = *s_chunk;
+  const long long total = (long long)Hkv * s_cum[n];          // pages of the static stream
+  const int n_static = a.n_static;                            // = gridDim.x * kWarps
+  const long long W = total > 0 ? (total + n_static - 1) / n_static : 1;
+  const int n_dyn = Hkv * s_cumc[n];                          // chunks to hand out
   const int part = blockIdx.x * kWarps + warp;
-  const long long pos0 = (long long)part * W;
-  if (W == 0 || pos0 >= total) {
-    before_first_write();
-    fill_empty_traces();
-    return;
-  }
-  const int cnt = (int)((pos0 + W <= total ? pos0 + W : total) - pos0);
 
-  unsigned char* my_pages = s_pages + (size_t)warp * kStages * kPageBytes;
-  const uint32_t my_pages_u32 = smem_u32(my_pages);
+  const uint32_t my_pages_u32 = smem_u32(s_pages + (size_t)warp * kStages * kPageBytes);
   const uint32_t my_bar_u32 = smem_u32(&s_bar[warp * kStages]);
+
+  // A unit of work: this warp's share of the static stream (idx = its partition, `cnt` pages from stream position
+  // pos0 on), or a chunk (idx = chunk number: pages p0 .. p0 + cnt - 1 of sequence (t, h)).
+  struct Unit { long long pos0; int cnt, idx, t, h, p0; bool chunk; };
+  Unit cur, nxt;
+  cur.chunk = false; cur.idx = part; cur.pos0 = (long long)part * W; cur.t = cur.h = cur.p0 = 0;
+  cur.cnt = cur.pos0 < total ? (int)((cur.pos0 + W <= total ? cur.pos0 + W : total) - cur.pos0) : 0;
+  nxt = cur;
+  bool have_nxt = false, dyn_done = n_dyn == 0;
 
   // ---- producer side: cursor, block-id window (lane i holds the id of page win_base + i)
   Cursor pc;
-  cursor_seek(pc, s_cum, n, Hkv, pos0);
+  bool p_chunk = false;
+  if (cur.cnt > 0) cursor_seek(pc, s_cum, n, Hkv, cur.pos0);
   int win_t = -1, win_base = 0, win_ids = 0;
-  int issued = 0;
-  auto produce = [&](int stage) {
+  int p_left = cur.cnt, p_stage = 0, in_flight = 0;
+  // the next chunk into nxt; false when none is left.  The counter is shared with the launch before this one (if
+  // this launch was scheduled ahead of that one's completion); the kernel that combines a launch's pieces puts it
+  // back to zero.
+  auto claim = [&]() -> bool {
+    if (dyn_done) return false;
+    before_first_write();
+    for (;;) {
+      int c = 0;
+      if (lane == 0) c = atomicAdd(&a.sched[0], 1);
+      c = __shfl_sync(0xffffffffu, c, 0);
+      if (c >= n_dyn) { dyn_done = true; return false; }
+      const int t = seek_trace(s_cumc, n, Hkv, c);
+      const int r = c - Hkv * s_cumc[t], ch = s_cumc[t + 1] - s_cumc[t];
+      const int j = r % ch;
+      if (j == ch - 1) continue;                       // the number that stands for no pages
+      nxt.chunk = true; nxt.idx = c; nxt.t = t; nxt.h = r / ch;
+      nxt.p0 = (s_cum[t + 1] - s_cum[t]) + j * C;
+      nxt.cnt = min(C, s_np[t] - nxt.p0);
+      nxt.pos0 = 0;
+      return true;
+    }
+  };
+  // one more page copy into the ring, if a slot is free and a page is left to fetch
+  auto issue_one = [&]() -> bool {
+    if (in_flight == kStages) return false;
+    if (p_left == 0) {
+      if (have_nxt || !claim()) return false;          // (the consumer has yet to enter the chunk claimed last)
+      have_nxt = true;
+      p_chunk = true;
+      pc.t = nxt.t; pc.h = nxt.h; pc.page = nxt.p0; pc.np = s_np[nxt.t];
+      p_left = nxt.cnt;
+      win_t = -1;
+    }
     if (pc.t != win_t || pc.page < win_base || pc.page >= win_base + 32) {
       win_t = pc.t; win_base = pc.page;
       const int pg = win_base + lane;
@@ -297,18 +412,21 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     if (lane == 0) {
       if (b < 0 || b >= a.num_blocks) { flag_error(a.counters, STEP_ERR_BAD_BLOCK); b = 0; }
       const __nv_bfloat16* src = a.kv_layer + ((size_t)b * Hkv + pc.h) * (size_t)(2 * kP * kD);
-      const uint32_t bar = my_bar_u32 + stage * 8;
+      const uint32_t bar = my_bar_u32 + p_stage * 8;
       mbar_expect_tx(bar, kPageBytes);
-      bulk_load(my_pages_u32 + stage * kPageBytes, src, kPageBytes, bar);
+      bulk_load(my_pages_u32 + p_stage * kPageBytes, src, kPageBytes, bar);
     }
-    cursor_next(pc, s_cum, n, Hkv);
-    ++issued;
+    if (p_chunk) ++pc.page; else cursor_next(pc, s_cum, n, Hkv);
+    --p_left; ++in_flight;
+    if (++p_stage == kStages) p_stage = 0;
+    return true;
   };
-  for (int s = 0; s < kStages && issued < cnt; ++s) produce(s);
+  while (issue_one()) {}
 
   // ---- consumer side
   Cursor cc;
-  cursor_seek(cc, s_cum, n, Hkv, pos0);
+  if (cur.cnt > 0) cursor_seek(cc, s_cum, n, Hkv, cur.pos0);
+  int c_left = cur.cnt;
   const int g_row = lane >> 2, tq = lane & 3;
   uint32_t qa[8][4];                 // A fragments of Q for the 8 k-steps over head_dim
   float o_acc[16][4];                // O fragments: 16 n-tiles over head_dim
@@ -318,7 +436,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   int stage = 0;
   uint32_t parity = 0;
   bool alive = true;
-  int timed_out_at = 0;
+  const int R = kMode == kPrefixPass ? 16 : G;         // rows of a partial slot
 
   // ldmatrix lane addressing inside a page (swizzled 16-byte chunks: chunk' = chunk ^ (row & 7))
   const int mi = lane >> 3, r8 = lane & 7;
@@ -327,7 +445,18 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   const int v_row = ((mi & 1) << 3) + r8;              // V: matrices 0,2 -> tokens 0-7; 1,3 -> tokens 8-15
   const int v_csel = mi >> 1;                          //    matrices 2,3 belong to the next 8-wide dim tile
 
-  for (int i = 0; i < cnt; ++i) {
+  for (;;) {
+    if (c_left == 0) {
+      // this unit is done: on to the chunk the producer has claimed (it claims one now if it had no reason to yet)
+      while (issue_one()) {}
+      if (!have_nxt) break;
+      cur = nxt; have_nxt = false;
+      cc.t = cur.t; cc.h = cur.h; cc.page = cur.p0; cc.np = s_np[cur.t];
+      c_left = cur.cnt;
+      seg_open = false; seg_is_first = true;
+    }
+    // pages of sequence cc.t in the static stream (a segment of a static share ends there at the latest)
+    const int np_static = s_cum[cc.t + 1] - s_cum[cc.t];
     if (!seg_open) {
       // new (trace, head) segment: Q fragments of the G heads of this group, fresh softmax state
       if (a.q_from_primary) before_first_write();
@@ -364,7 +493,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     if (!mbar_wait_bounded(my_bar_u32 + stage * 8, parity, a.wait_ns)) {
       if (lane == 0) flag_error(a.counters, STEP_ERR_TIMEOUT);
       alive = false;
-      timed_out_at = i;
       break;
     }
     const uint32_t kpage = my_pages_u32 + stage * kPageBytes;
@@ -372,7 +500,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
     // tokens of this page that exist (only the last page of a sequence can be short)
     int valid = kP;
-    if (kMode != kPrefixPass && cc.page == cc.np - 1) {    // shared pages are full
+    if (kMode != kPrefixPass && cc.page == s_np[cc.t] - 1) {    // shared pages are full
       int S = a.seq_lens[cc.t];
       const int cap = a.max_pages * kP;
       if (S > cap) S = cap;
@@ -451,10 +579,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
       mma_bf16(o_acc[2 * dp + 1], pa0, pa1, pa2, pa3, b2, b3);
     }
     __syncwarp();
-    if (issued < cnt) produce(stage);                  // refill the stage just consumed
+    --in_flight;
+    while (issue_one()) {}                             // refill the stage just consumed
 
     // ---- end of this (trace, head) segment?
-    const bool seg_end = (cc.page + 1 == cc.np) || (i + 1 == cnt);
+    const bool seq_static_end = !cur.chunk && cc.page + 1 == np_static;
+    const bool seg_end = seq_static_end || c_left == 1;
     if (seg_end) {
       float l0 = l_run[0];
       l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
@@ -464,8 +594,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
       }
-      const bool complete = seg_first_page == 0 && cc.page + 1 == cc.np;
-      const int R = kMode == kPrefixPass ? 16 : G;       // rows of a partial slot
+      // the whole sequence in this one segment: it has no tail, and its static pages lie in this share
+      const bool complete = seq_static_end && seg_first_page == 0 && np_static == s_np[cc.t];
       before_first_write();
       if (complete && kMode == kPrefixPass) {
         // the bundle's whole prefix was read by this warp: (m, l, o) of every (trace, head) row, un-normalised
@@ -531,7 +661,22 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
           }
         }
       } else {
-        const size_t slot = (size_t)part * 2 + (seg_is_first ? 0 : 1);
+        // ---- a piece of a sequence: leave its (m, l, o) in this piece's slot.
+        // The sequence's chunk numbers are cbase .. cbase + n_ch (n_ch chunks, then the number that stands for no
+        // pages); its static part lies in shares s0p .. s1p.  A static piece that reaches an
+        // edge of its share uses one of the share's two slots (every share has at most one piece at each edge); a
+        // static part that lies inside a single share - there may be many of those in one share - uses the slot of
+        // the sequence's spare chunk number.  (A sequence without a tail whose static part lies inside one share
+        // was complete and never gets here.)
+        const int n_nums = s_cumc[cc.t + 1] - s_cumc[cc.t];
+        const int n_ch = n_nums > 0 ? n_nums - 1 : 0;
+        const int cbase = Hkv * s_cumc[cc.t] + cc.h * n_nums;
+        const long long seg_start = (long long)Hkv * s_cum[cc.t] + (long long)cc.h * np_static;
+        const int s0p = (int)(seg_start / W), s1p = (int)((seg_start + np_static - 1) / W);
+        const int n_s = s1p - s0p + 1;
+        const size_t spare = (size_t)kDynSlotBase + cbase + n_ch;
+        const size_t slot = cur.chunk ? (size_t)kDynSlotBase + cur.idx
+                                      : (n_s == 1 ? spare : (size_t)cur.idx * 2 + (seg_is_first ? 0 : 1));
         float* ml = a.ws_ml + slot * R * 2;
         float* ob = a.ws_o + slot * R * kD;
         if (g_row < R) {
@@ -546,90 +691,165 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
           for (int dt = 0; dt < 16; ++dt)
             *reinterpret_cast<float2*>(ob + (size_t)(g_row + 8) * kD + dt * 8 + 2 * tq) = make_float2(o_acc[dt][2], o_acc[dt][3]);
         }
-        // publish the partial, take a ticket; the last of the sequence's partitions to arrive merges them all
-        __threadfence();
-        __syncwarp();
-        const long long seg_start = (long long)Hkv * s_cum[cc.t] + (long long)cc.h * cc.np;
-        const int w_first = (int)(seg_start / W), w_last = (int)((seg_start + cc.np - 1) / W);
-        int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&a.seg_cnt[cc.t * Hkv + cc.h], 1);
-        ticket = __shfl_sync(0xffffffffu, ticket, 0);
-        if (ticket == w_last - w_first) {
-          if (lane == 0) a.seg_cnt[cc.t * Hkv + cc.h] = 0;             // ready for the next launch
-          __threadfence();
-          const int rows = kMode == kPrefixPass ? a.tpb * G : G;
-          for (int g = 0; g < rows; ++g) {
-            size_t idx = 0;                                            // (trace, head) row of pre_ml / pre_o
-            if constexpr (kMode == kPrefixPass) {
-              const int t = cc.t * a.tpb + g / G;
-              if (t >= a.n) break;
-              idx = (size_t)t * a.Hq + (size_t)cc.h * G + g % G;
-            } else if constexpr (kMode == kSuffixPass) {
-              idx = (size_t)cc.t * a.Hq + (size_t)cc.h * G + g;
-            }
-            float M = kMode == kSuffixPass ? a.pre_ml[idx * 2] : -INFINITY;
-            for (int w = w_first; w <= w_last; ++w) {
-              const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
-              M = fmaxf(M, __ldcg(&a.ws_ml[(sl * R + g) * 2]));
-            }
-            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-            float den = 0.f;
-            if constexpr (kMode == kSuffixPass) {                      // the shared pages count as one more partial
-              const float wgt = exp2f(a.pre_ml[idx * 2] - M);
-              den = wgt * a.pre_ml[idx * 2 + 1];
-              const float4 o4 = reinterpret_cast<const float4*>(a.pre_o + idx * kD)[lane];
-              num = make_float4(wgt * o4.x, wgt * o4.y, wgt * o4.z, wgt * o4.w);
-            }
-            for (int w = w_first; w <= w_last; ++w) {
-              const size_t sl = (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
-              const float wgt = exp2f(__ldcg(&a.ws_ml[(sl * R + g) * 2]) - M);
-              den += wgt * __ldcg(&a.ws_ml[(sl * R + g) * 2 + 1]);
-              const float4 o4 = __ldcg(reinterpret_cast<const float4*>(a.ws_o + (sl * R + g) * kD) + lane);
-              num.x += wgt * o4.x; num.y += wgt * o4.y; num.z += wgt * o4.z; num.w += wgt * o4.w;
-            }
-            if constexpr (kMode == kPrefixPass) {
-              if (lane == 0) { a.pre_ml[idx * 2] = M; a.pre_ml[idx * 2 + 1] = den; }
-              reinterpret_cast<float4*>(a.pre_o + idx * kD)[lane] = num;
-            } else {
-              float* og = a.out + ((size_t)cc.t * a.Hq + (size_t)cc.h * G) * kD;
-              const float inv = 1.f / den;
-              reinterpret_cast<float4*>(og + (size_t)g * kD)[lane] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
-            }
-          }
-        }
       }
       seg_open = false;
       seg_is_first = false;
     }
-    cursor_next(cc, s_cum, n, Hkv);
+    if (cur.chunk) ++cc.page; else cursor_next(cc, s_cum, n, Hkv);
+    --c_left;
     if (++stage == kStages) { stage = 0; parity ^= 1; }
   }
 
   before_first_write();
   fill_empty_traces();
   if (!alive) {
-    // A wait ran out.  The copies of pages timed_out_at .. issued - 1 were issued and still target this CTA's shared
-    // memory: each gets one more wait, with the full limit, before the warp leaves (page j uses stage j % kStages in
-    // the phase of parity (j / kStages) & 1); nothing else is touched.
-    for (int j = timed_out_at; j < issued; ++j)
-      mbar_wait_bounded(my_bar_u32 + (j % kStages) * 8, (uint32_t)((j / kStages) & 1));
+    // A wait ran out.  The in_flight copies issued last still target this CTA's shared memory (ring positions stage,
+    // stage + 1, ... in the consumer's order): each gets one more wait, with the full limit, before the warp
+    // leaves; nothing else is touched.
+    for (int k = 0; k < in_flight; ++k) {
+      const int st = stage + k;
+      mbar_wait_bounded(my_bar_u32 + (st % kStages) * 8, parity ^ (uint32_t)(st >= kStages));
+    }
+  }
+}
+
+// Combines, for every (sequence, KV head) of the launch that was cut into pieces, the pieces' partials into the
+// output (or, for the shared pages' pass, into that pass's result).  Work item = one query row of one sequence's
+// tile, taken by one warp (items are dealt round-robin to all warps of the grid): the warp takes the row's pieces in
+// stream order - static pieces, then chunks - eight at a time (all their loads issued together: one round trip to
+// memory for most sequences), lanes over the 128 dims, and keeps a running (max, sum, weighted values) across the
+// batches; a fixed order, so the same bits whatever ran where.
+// Launched as a programmatic dependent of the attention kernel, with at most one small CTA per SM and few enough
+// registers that it is resident BESIDE the attention kernel's CTA: it works out where the pieces are from the
+// launch's lengths - the same functions the attention kernel uses - while that kernel is still running, then waits
+// for it.  (A launch chained behind this one is scheduled only when every CTA of this one has started, so CTAs that
+// had to queue for an SM would hold back the next layer's launch until this layer is over.)
+constexpr int kMergeBatch = 8, kMergeWarps = 4;
+
+template <int kMode>
+__global__ void __launch_bounds__(kMergeWarps * 32, 5) attn_merge_kernel(AttnArgs a) {
+  extern __shared__ int s_part[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int Hkv = a.Hkv, G = a.G;
+  const int R = kMode == kPrefixPass ? 16 : G;                    // rows of a partial slot
+  const int rows = kMode == kPrefixPass ? a.tpb * G : G;          // rows in use
+  dependents_may_launch();
+  const int n = kMode == kPrefixPass ? a.n_bundles : a.n;
+  int* s_np = s_part;
+  int* s_cum = s_np + n;
+  int* s_cumc = s_cum + n + 1;
+  int* s_chunk = s_cumc + n + 1;
+  if (warp == 0) build_partition<kMode>(a, n, lane, false, s_np, s_cum, s_cumc, s_chunk);
+  __syncthreads();
+  const long long total = (long long)Hkv * s_cum[n];
+  const long long W = total > 0 ? (total + a.n_static - 1) / a.n_static : 1;
+
+  wait_for_primary();
+  if (blockIdx.x == 0 && threadIdx.x == 0 && a.sched) a.sched[0] = 0;   // the chunk counter, for the next launch
+
+  const int n_items = n * Hkv * rows;
+  for (int item = blockIdx.x * kMergeWarps + warp; item < n_items; item += gridDim.x * kMergeWarps) {
+    const int g = item % rows, th = item / rows;
+    const int t = th / Hkv, h = th - t * Hkv;
+    const int np_static = s_cum[t + 1] - s_cum[t];
+    if (np_static == 0) continue;                                 // no pages: the attention kernel wrote zeros
+    const int n_nums = s_cumc[t + 1] - s_cumc[t];
+    const int n_ch = n_nums > 0 ? n_nums - 1 : 0;
+    const int cbase = Hkv * s_cumc[t] + h * n_nums;
+    const long long seg_start = (long long)Hkv * s_cum[t] + (long long)h * np_static;
+    const int s0p = (int)(seg_start / W), s1p = (int)((seg_start + np_static - 1) / W);
+    const int n_s = s1p - s0p + 1;
+    const int n_pieces = n_s + n_ch;
+    if (n_pieces == 1) continue;                                  // one piece: the attention kernel wrote the output itself
+    const size_t spare = (size_t)kDynSlotBase + cbase + n_ch;
+    auto slot_of = [&](int k) -> size_t {
+      if (k < n_s) {
+        if (n_s == 1) return spare;
+        const int w = s0p + k;
+        return (size_t)w * 2 + (seg_start <= (long long)w * W ? 0 : 1);
+      }
+      return (size_t)kDynSlotBase + cbase + (k - n_s);
+    };
+    size_t idx = 0;                                               // (trace, head) row of pre_ml / pre_o
+    if constexpr (kMode == kPrefixPass) {
+      const int tt = t * a.tpb + g / G;
+      if (tt >= a.n) continue;
+      idx = (size_t)tt * a.Hq + (size_t)h * G + g % G;
+    } else if constexpr (kMode == kSuffixPass) {
+      idx = (size_t)t * a.Hq + (size_t)h * G + g;
+    }
+
+    float M = -INFINITY, den = 0.f;
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k0 = 0; k0 < n_pieces; k0 += kMergeBatch) {
+      float2 ml[kMergeBatch];
+      float4 o4[kMergeBatch];
+#pragma unroll
+      for (int j = 0; j < kMergeBatch; ++j) {
+        if (k0 + j < n_pieces) {
+          const size_t sl = slot_of(k0 + j);
+          ml[j] = __ldcg(reinterpret_cast<const float2*>(a.ws_ml + (sl * R + g) * 2));
+          o4[j] = __ldcg(reinterpret_cast<const float4*>(a.ws_o + (sl * R + g) * kD) + lane);
+        }
+      }
+      float Mb = M;
+#pragma unroll
+      for (int j = 0; j < kMergeBatch; ++j)
+        if (k0 + j < n_pieces) Mb = fmaxf(Mb, ml[j].x);
+      const float keep = exp2f(M - Mb);                           // 0 on the first batch (M = -inf)
+      den *= keep; num.x *= keep; num.y *= keep; num.z *= keep; num.w *= keep;
+      M = Mb;
+#pragma unroll
+      for (int j = 0; j < kMergeBatch; ++j) {
+        if (k0 + j < n_pieces) {
+          const float wgt = exp2f(ml[j].x - M);
+          den += wgt * ml[j].y;
+          num.x += wgt * o4[j].x; num.y += wgt * o4[j].y; num.z += wgt * o4[j].z; num.w += wgt * o4[j].w;
+        }
+      }
+    }
+    if constexpr (kMode == kSuffixPass) {                         // the shared pages count as one more partial
+      const float mp = a.pre_ml[idx * 2], lp = a.pre_ml[idx * 2 + 1];
+      const float4 o4 = reinterpret_cast<const float4*>(a.pre_o + idx * kD)[lane];
+      const float Mb = fmaxf(M, mp);
+      const float keep = exp2f(M - Mb), wgt = exp2f(mp - Mb);
+      den = den * keep + wgt * lp;
+      num.x = num.x * keep + wgt * o4.x; num.y = num.y * keep + wgt * o4.y;
+      num.z = num.z * keep + wgt * o4.z; num.w = num.w * keep + wgt * o4.w;
+    }
+    if constexpr (kMode == kPrefixPass) {
+      if (lane == 0) { a.pre_ml[idx * 2] = M; a.pre_ml[idx * 2 + 1] = den; }
+      reinterpret_cast<float4*>(a.pre_o + idx * kD)[lane] = num;
+    } else {
+      float* og = a.out + ((size_t)t * a.Hq + (size_t)h * G + g) * kD;
+      const float inv = 1.f / den;
+      reinterpret_cast<float4*>(og)[lane] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+    }
   }
 }
 
 constexpr int kWarpsDefault = 8, kStagesDefault = 3;
 
-// dependent: the launch may be scheduled before the kernel ahead of it in the stream has completed (see the kernel's
-// note on its first write); only for a launch that directly follows another launch of this kernel on the same pool.
+// The attention kernel, then the kernel that combines its pieces as its programmatic dependent.
+// dependent: the attention launch itself may be scheduled before the kernel ahead of it in the stream has completed
+// (see the kernel's note on its first write).
 template <int kWarps, int kStages, bool kRows16, int kMode>
-int launch_one(const AttnArgs& a, int grid, cudaStream_t s, bool dependent = false) {
-  const size_t smem = (size_t)kWarps * kStages * kPageBytes + (size_t)kWarps * kStages * 8 + (size_t)(a.n + 1) * 4;
+int launch_one(AttnArgs a, int grid, cudaStream_t s, bool dependent = false) {
+  const int n_seq = kMode == kPrefixPass ? a.n_bundles : a.n;
+  const size_t smem = (size_t)kWarps * kStages * kPageBytes + (size_t)kWarps * kStages * 8 + (size_t)(3 * n_seq + 3) * 4;
+  a.n_static = grid * kWarps;
   auto kern = attn_mma_kernel<kWarps, kStages, kRows16, kMode>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return STEP_ERR_CUDA;
   if (dependent) {
     if (launch_dependent(kern, dim3(grid), dim3(kWarps * 32), smem, s, a) != cudaSuccess) return STEP_ERR_CUDA;
   } else {
     kern<<<grid, kWarps * 32, smem, s>>>(a);
+    if (launch_ok() != STEP_OK) return STEP_ERR_CUDA;
   }
+  const int rows = kMode == kPrefixPass ? a.tpb * a.G : a.G;
+  long long mgrid = ((long long)n_seq * a.Hkv * rows + kMergeWarps - 1) / kMergeWarps;
+  if (mgrid > a.merge_ctas) mgrid = a.merge_ctas;
+  if (launch_dependent(attn_merge_kernel<kMode>, dim3((int)mgrid), dim3(kMergeWarps * 32), (size_t)(3 * n_seq + 3) * 4, s, a) != cudaSuccess) return STEP_ERR_CUDA;
   return launch_ok();
 }
 
@@ -647,11 +867,15 @@ void fill_args(AttnArgs& a, const step_pool* pool, const Geo& g, int layer, cons
   a.kv_layer = (const __nv_bfloat16*)pool->cfg.kv_storage + (size_t)layer * g.num_blocks * g.Hkv * 2 * kP * kD;
   a.q = (const __nv_bfloat16*)q;
   a.block_table = block_table; a.seq_lens = seq_lens; a.out = (float*)out;
-  a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.seg_cnt = pool->v.attn_cnt; a.counters = pool->v.counters;
+  a.ws_ml = pool->v.attn_ml; a.ws_o = pool->v.attn_o; a.counters = pool->v.counters;
   a.n = n; a.Hq = g.Hq; a.Hkv = g.Hkv; a.G = g.G; a.max_pages = g.max_pages; a.num_blocks = g.num_blocks;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.d);
   a.prefix_blocks = nullptr; a.pre_ml = nullptr; a.pre_o = nullptr; a.pp = 0; a.tpb = 1; a.n_bundles = 0;
   a.q_from_primary = 0;
+  a.sched = pool->attn_dyn16 > 0 ? pool->v.attn_sched : nullptr;
+  a.dyn16 = pool->attn_dyn16; a.dyn_chunk = pool->attn_dyn_chunk;
+  a.n_static = 0;                                      // set by the launcher
+  a.merge_ctas = pool->num_sms;
   a.wait_ns = pool->wait_limit_ns;
 }
 
@@ -757,6 +981,7 @@ extern "C" int decode_attention_shared_prefix(step_pool* pool, int layer, const 
   // pass 1: about eight pages per warp, at most one CTA per SM and kPrefixPartitions partitions
   AttnArgs p1 = a;
   p1.ws_ml = pool->v.pre_ws_ml; p1.ws_o = pool->v.pre_ws_o;
+  p1.sched = nullptr;                                  // its scratch holds equal shares only
   const long long pages1 = (long long)a.n_bundles * g.Hkv * prefix_pages;
   long long grid1 = (pages1 + kWarpsDefault * 8 - 1) / (kWarpsDefault * 8);
   const int cap1 = pool->attn_grid < kPrefixPartitions / kWarpsDefault ? pool->attn_grid : kPrefixPartitions / kWarpsDefault;
@@ -790,8 +1015,8 @@ constexpr int kStaticMaxPartitions = 1184;   // 148 SMs x 8 warps
 constexpr int kStaticMaxG = 8;               // query heads per KV head
 constexpr size_t kStaticMlFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * 2;
 constexpr size_t kStaticOFloats = (size_t)kStaticMaxPartitions * 2 * kStaticMaxG * kD;
-constexpr int kStaticMaxSegs = 16384;        // (trace, KV head) sequences of one call: their ticket counters
-constexpr size_t kStaticScratchFloats = kStaticMlFloats + kStaticOFloats + kStaticMaxSegs;
+constexpr int kStaticMaxSegs = 16384;        // (trace, KV head) sequences of one call
+constexpr size_t kStaticScratchFloats = kStaticMlFloats + kStaticOFloats;
 
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
@@ -835,13 +1060,9 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   if (grid < 1) grid = 1;
   AttnArgs a;
   fill_args(a, pool, g, layer, q, block_table, seq_lens, n, out);
-  // the same kernel, its partials and tickets in the library's own array instead of the pool's metadata
+  // the same kernels, the partials in the library's own array instead of the pool's metadata
   a.ws_ml = scratch; a.ws_o = scratch + kStaticMlFloats;
-  a.seg_cnt = reinterpret_cast<int32_t*>(scratch + kStaticMlFloats + kStaticOFloats);
+  a.sched = nullptr;                                   // the fixed array holds the partials of equal shares only
   cudaStream_t s = (cudaStream_t)stream;
-  // The tickets of this call's (trace, KV head) sequences must start at zero.  A call that runs to its end leaves
-  // them zero, but one whose bounded wait ran out does not, and nothing else ever resets this array: clear them on
-  // the stream first (a memset of at most 64 KiB; no allocation).
-  STEP_CUDA_OK(cudaMemsetAsync(a.seg_cnt, 0, (size_t)n * g.Hkv * sizeof(int32_t), s));
   return launch_one<kWarpsDefault, kStagesDefault, false, kPlain>(a, grid, s);
 }

@@ -51,11 +51,13 @@ MetaLayout make_layout(const kv_pool_config* c) {
   l.score_z = take(rows * kScoreSplits * 4);
   l.score_part = take((rows + kScoreFoldRows - 1) / kScoreFoldRows * T * 8);
   l.score_zs = take((size_t)kSmallRows * kSmallCtas * 4);
-  l.attn_ml = take((size_t)kMaxPartitions * 2 * G * 2 * 4);
-  l.attn_o = take((size_t)kMaxPartitions * 2 * G * c->head_dim * 4);
-  l.attn_cnt = take((size_t)kMaxTracesFast * c->num_kv_heads * 4);
-  // shared-prefix attention: partials of its first pass (16 query rows per slot) and that pass's result per (trace, head)
+  // attention partials: two slots per equal share, then (tensor-core shape only) one per chunk handed out at run time
   const bool mma = c->dtype == STEP_BF16 && c->head_dim == 128 && c->page_size == 16;
+  const size_t slots = (size_t)kMaxPartitions * 2 + (mma ? kMaxDynChunks : 0);
+  l.attn_ml = take(slots * G * 2 * 4);
+  l.attn_o = take(slots * G * c->head_dim * 4);
+  l.attn_sched = take(4);
+  // shared-prefix attention: partials of its first pass (16 query rows per slot) and that pass's result per (trace, head)
   l.pre_ws_ml = take(mma ? (size_t)kPrefixPartitions * 2 * 16 * 2 * 4 : 0);
   l.pre_ws_o = take(mma ? (size_t)kPrefixPartitions * 2 * 16 * c->head_dim * 4 : 0);
   l.pre_ml = take(mma ? T * c->num_q_heads * 2 * 4 : 0);
@@ -92,7 +94,7 @@ __global__ void init_meta_kernel(DevViews v, Geo g, float unscored) {
     v.free_list[i] = g.num_blocks - 1 - (int)i;       // a stack: the first pop is block 0
   }
   for (size_t i = tid; i < (size_t)C_NUM; i += stride) v.counters[i] = (i == C_FREE_COUNT) ? g.num_blocks : 0;
-  for (size_t i = tid; i < (size_t)kMaxTracesFast * g.Hkv; i += stride) v.attn_cnt[i] = 0;
+  if (tid == 0) v.attn_sched[0] = 0;
 }
 
 // ---------------------------------------------------------------- InitTraces (fork)
@@ -372,6 +374,8 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->max_score_rows = cfg->max_score_rows > 0 ? cfg->max_score_rows : cfg->max_traces;
   p->num_sms = sms;
   p->attn_grid = sms;
+  p->attn_dyn16 = 4;
+  p->attn_dyn_chunk = 16;
   p->fast_path = 1;
   p->wait_limit_ns = 2000000000ull;
   p->scorer_mode = 0;
@@ -391,7 +395,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   v.score_idx = (int32_t*)(m + lay.score_idx); v.score_z = (float*)(m + lay.score_z);
   v.score_part = (float2*)(m + lay.score_part);
   v.score_zs = (float*)(m + lay.score_zs);
-  v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o); v.attn_cnt = (int32_t*)(m + lay.attn_cnt);
+  v.attn_ml = (float*)(m + lay.attn_ml); v.attn_o = (float*)(m + lay.attn_o); v.attn_sched = (int32_t*)(m + lay.attn_sched);
   const bool mma = lay.pre_ws_o != lay.pre_ml;      // the regions are zero-sized for other shapes
   v.pre_ws_ml = mma ? (float*)(m + lay.pre_ws_ml) : nullptr; v.pre_ws_o = mma ? (float*)(m + lay.pre_ws_o) : nullptr;
   v.pre_ml = mma ? (float*)(m + lay.pre_ml) : nullptr; v.pre_o = mma ? (float*)(m + lay.pre_o) : nullptr;
@@ -572,6 +576,13 @@ int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path) 
   if (!pool || grid_ctas < 0) return STEP_ERR_INVALID_ARG;
   if (grid_ctas > 0) pool->attn_grid = grid_ctas;
   if (fast_path != 0) pool->fast_path = fast_path > 0 ? 1 : -1;
+  return STEP_OK;
+}
+
+int kv_pool_set_attention_balance(step_pool* pool, int dynamic_sixteenths, int min_chunk_pages) {
+  if (!pool || dynamic_sixteenths < 0 || dynamic_sixteenths > 12 || min_chunk_pages < 0) return STEP_ERR_INVALID_ARG;
+  pool->attn_dyn16 = dynamic_sixteenths;
+  if (min_chunk_pages > 0) pool->attn_dyn_chunk = min_chunk_pages;
   return STEP_OK;
 }
 

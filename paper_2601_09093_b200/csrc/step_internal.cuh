@@ -21,6 +21,7 @@ namespace stepk {
 
 constexpr int kMaxPartitions = 4096;   // upper bound on independent KV-stream partitions of one launch
 constexpr int kPrefixPartitions = 1184; // partitions of the shared-prefix pass of decode_attention_shared_prefix (148 SMs x 8 warps)
+constexpr int kMaxDynChunks = 8192;    // upper bound on the chunks of one attention launch handed out at run time (partial slots beyond those of the shares)
 constexpr int kMaxTracesFast = 2048;   // traces per decode_attention call on the tensor-core path
 constexpr int kScoreSplits = 16;       // slices of the scorer's hidden units; score_z holds this many floats per row
 constexpr int kSmallRows = 256;       // candidate rows up to which score_steps is one launch (a decode step's shape)
@@ -44,7 +45,7 @@ struct MetaLayout {
   size_t refcount, free_list, claim, counters;
   size_t append_base, prune_rank, prune_list, prune_off;
   size_t score_idx, score_z, score_part, score_zs;
-  size_t attn_ml, attn_o, attn_cnt;
+  size_t attn_ml, attn_o, attn_sched;
   size_t pre_ws_ml, pre_ws_o, pre_ml, pre_o;   // shared-prefix attention (zero-sized for pools the tensor-core kernel does not cover)
   size_t final_score, answer, finished, it_ids, it_fin, it_pruned, it_tokens, it_scores;
   size_t total;
@@ -56,7 +57,7 @@ struct DevViews {
   int32_t* refcount; int32_t* free_list; int32_t* claim; int32_t* counters;
   int32_t* append_base; int32_t* prune_rank; int32_t* prune_list; int32_t* prune_off;
   int32_t* score_idx; float* score_z; float2* score_part; float* score_zs;
-  float* attn_ml; float* attn_o; int32_t* attn_cnt;
+  float* attn_ml; float* attn_o; int32_t* attn_sched;
   float* pre_ws_ml; float* pre_ws_o; float* pre_ml; float* pre_o;   // null when zero-sized
   float* final_score; int32_t* answer; uint8_t* finished;     // traces that completed: what the vote needs
   int32_t* it_ids; int32_t* it_fin; int32_t* it_pruned;       // per-iteration lists of the Algorithm 1 driver
@@ -73,6 +74,8 @@ struct step_pool {
   int max_score_rows;
   int num_sms;
   int attn_grid;      // CTAs of the tensor-core attention launch
+  int attn_dyn16;     // sixteenths of every sequence's pages handed out at run time (0: equal shares only)
+  int attn_dyn_chunk; // smallest chunk handed out, in pages
   int fast_path;      // 1 allowed, -1 forced off
   unsigned long long wait_limit_ns;   // limit of decode_attention's wait for a page copy (kv_pool_set_wait_limit_ns)
   int scorer_mode;    // 0: tensor-core MLP for launches with >= scorer_tc_min_rows boundary rows; 1: always; -1: never

@@ -235,6 +235,37 @@ def test_attention_grid_sizes_and_page_shuffle_agree():
     assert np.abs(outs[0] - outs[5]).max() < 1e-5      # only the physical placement differs
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (16, 1)])
+def test_attention_is_the_same_however_the_pages_are_handed_out(Hq, Hkv):
+    """Equal shares only, the default, and up to three quarters of every sequence in chunks of one page and more
+    (hundreds of chunks, fetched by whichever warp is free): every setting within tolerance of the oracle, a
+    setting's repeat bit-identical, and the shared-prefix call under the same settings too."""
+    cfg = W.scaled(W.C1, n_traces=9, num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=96)
+    suffix = [0, 1, 15, 16, 17, 700, 2049, 333, 5000]
+    tw, ids = _build(cfg, suffix)
+    qb, qx = W.normal(cfg.seed, W.TID_Q, (9, Hq, 128), "bf16")
+    qd = H.to_device(qb, "bf16")
+    want = _oracle_attention(tw, 0, qx, 9)
+    v = tw.gpu.views()
+    pp = 96 // 16
+    prefix_blocks = v["block_table"][0, :pp].clone()
+    with pytest.raises(Exception):
+        tw.gpu.set_attention_balance(13)
+    for grid in (0, 5):
+        tw.gpu.set_attention_config(grid_ctas=grid)
+        for sixteenths, chunk in [(0, 0), (4, 16), (4, 1), (12, 1), (12, 3), (8, 64)]:
+            tw.gpu.set_attention_balance(sixteenths, chunk)
+            got = exact_f32(_gpu_attention(tw, 0, qd, 9))
+            mx, mean = attention_errors(got, want)
+            assert mx <= ATT_MAX and mean <= ATT_MEAN, (grid, sixteenths, chunk, mx, mean)
+            again = exact_f32(_gpu_attention(tw, 0, qd, 9))
+            assert np.array_equal(got, again), (grid, sixteenths, chunk)
+            out = tw.gpu.decode_attention_shared_prefix(0, qd, v["block_table"][:9], v["seq_lens"][:9], prefix_blocks, pp)
+            mx, mean = attention_errors(exact_f32(out), want)
+            assert mx <= ATT_MAX and mean <= ATT_MEAN, ("shared prefix", grid, sixteenths, chunk, mx, mean)
+    assert tw.status() == (0, 0)
+
+
 def test_attention_padding_slots_do_not_leak():
     # unused slots of the last page hold NaN bit patterns: the result must not see them
     cfg = W.scaled(W.C1, n_traces=2, prefix_len=0)
