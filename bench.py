@@ -38,7 +38,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer", "prefix", "replay"])
+    ap.add_argument("--workload", default="c3", choices=["c3", "c1", "c2", "c4", "scorer", "prefix", "replay", "append"])
     ap.add_argument("--prefix-len", type=int, default=8192, help="prefix workload: tokens of the shared prompt")
     ap.add_argument("--suffix-max", type=int, default=512, help="prefix workload: traces hold 1 .. this many tokens of their own")
     ap.add_argument("--scorer-rows", type=int, default=65536, help="rows of the batched scorer workload")
@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--no-aux", action="store_true", help="skip the scorer / prune-cycle measurements after the timed steps")
     ap.add_argument("--num-blocks", type=int, default=0, help="override the pool size (blocks)")
     ap.add_argument("--grid", type=int, default=0, help="CTAs of the attention launch (0 = library default)")
+    ap.add_argument("--balance", type=int, default=-1,
+                    help="sixteenths of every sequence's pages that the attention launches of the timed steps hand out at run "
+                         "time (kv_pool_set_attention_balance); -1 = 2 when a step chains several layers' launches, else the library's 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -207,6 +210,12 @@ def run_ours(args):
     pool = H.make_pool(cfg_pool, nb, max_pages, T, max_score_rows=T, device=dev)
     if args.grid:
         pool.set_attention_config(grid_ctas=args.grid)
+    # In a chain of launches (decode_attention_layers) an SM that is done early starts on the next layer, so less of
+    # the stream needs handing out at run time than for a launch on its own: measured on one device, 36-layer steps
+    # took 21.29 / 20.59 / 20.76 / 20.85 ms with 0 / 2 / 4 / 6 sixteenths, one-layer steps 0.489 / 0.464 / 0.451 / 0.456 ms.
+    LIB_BALANCE = 4
+    step_balance = args.balance if args.balance >= 0 else (2 if L > 1 else LIB_BALANCE)
+    pool.set_attention_balance(step_balance)
     if cfg.shuffle_pages:
         H.shuffle_free_list(pool, cfg.seed + rank)
     t_fill = time.time()
@@ -374,7 +383,9 @@ def run_ours(args):
     attn_run_ms = [a.elapsed_time(b) for a, b, _ in attn_events]
     attn_ms = [t / nl for t, (_, _, nl) in zip(attn_run_ms, attn_events)]     # per launch, within its run of layers
     attn_launches = sum(nl for _, _, nl in attn_events)
-    # the same kernel launched alone (plain decode_attention calls, one event pair each), for comparison
+    # the same kernel launched alone (plain decode_attention calls, one event pair each), for comparison; launches
+    # on their own get the library's default balance
+    pool.set_attention_balance(LIB_BALANCE)
     iso = []
     for i in range(2 + 12):                                              # two untimed launches first
         l = i % phys_layers
@@ -386,13 +397,16 @@ def run_ours(args):
             iso.append((e0, e1))
     torch.cuda.synchronize()
     iso_ms = float(np.mean([a.elapsed_time(b) for a, b in iso]))
+    pool.set_attention_balance(step_balance)
     # whole steps the way a layer-by-layer engine would make them (outside `value`; single-GPU runs only)
     per_layer_ms = dep_layer_ms = prod_layer_ms = None
     probe = None
     if world == 1 and not args.no_aux:
+        pool.set_attention_balance(LIB_BALANCE)                          # one call per layer: launches on their own
         per_layer_ms = timed_steps(K, layer_calls="plain")
         prod_layer_ms = timed_steps(K, layer_calls="plain_after_producer")
         dep_layer_ms = timed_steps(K, layer_calls="dependent")
+        pool.set_attention_balance(step_balance)
         probe = read_stream_ceiling(pool, cfg, dev, L)
     err_code, err_mask = pool.last_error()
     n_live = pool.stats()["live_traces"]
@@ -442,6 +456,9 @@ def run_ours(args):
                    "page": cfg.page_size, "num_blocks": nb, "pool_gb": round(pool.kv_bytes / 1e9, 2),
                    "tokens_per_trace": int(np.mean(seq_now)), "threshold": cfg.threshold, "keep_frac": cfg.keep_frac,
                    "l2_policy": "inputs larger than L2 (%.1f GB of KV per layer call)" % (kv_bytes / 1e9),
+                   "attention_balance": {"timed_steps_sixteenths": step_balance, "single_launches_sixteenths": LIB_BALANCE,
+                                         "what": "share of every sequence's pages that warps fetch at run time "
+                                                 "(kv_pool_set_attention_balance); the rest is dealt out in equal shares"},
                    "multi_gpu": "replicas only (one independent problem per GPU)", "fill_s": round(t_fill, 1)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -684,7 +701,7 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     code, bits = pool.last_error()
     return {"iterations": r["iterations"], "ms_per_iteration": ms, "trace_decode_steps_per_s": T / (ms * 1e-3),
             "vs_python_driven_step": None if ms_per_step_python is None else ms_per_step_python / ms,
-            "layers_per_iteration": phys_layers, "launches_per_iteration": 4 + phys_layers,
+            "layers_per_iteration": phys_layers, "launches_per_iteration": 4 + 2 * phys_layers,
             "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
             "recorded_iterations": {"iterations": rg["iterations"], "ms_per_iteration": ms_g,
                                     "trace_decode_steps_per_s": T / (ms_g * 1e-3), "vs_direct_launches": ms / ms_g,
@@ -1030,6 +1047,28 @@ def run_scorer(args):
 
 
 # ---------------------------------------------------------------------------------------------
+def run_append(args):
+    """`--workload append`: append_kv alone - the 64-trace, 36-layer layout; `--steps` calls of each kind are timed
+    (the pool grows with that number: 2 steps hold 4 GB, the default 20 hold 10 GB)."""
+    import torch
+    from paper_2601_09093_b200 import ranks as R, workloads as W
+    from paper_2601_09093_b200 import build as _build
+    rank, local_rank, world = R.rank_env()
+    if rank != 0:
+        return
+    _build.build()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    m = append_measurements(W.C3, dev, W.C3.num_layers, reps=max(args.steps, 2))
+    b = m["bulk_32_tokens"]
+    print(json.dumps({"metric": "append_kv_bulk_bytes_per_s", "value": b["gbs"], "unit": "GB/s", "n_gpus": 1, "steps": max(args.steps, 2),
+                      "warmup": 3, "ms_per_step": b["us_per_call_device"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded, drawn on device)",
+                      "config": {"workload": "append_kv on the 64-trace 36-layer layout", "l2_policy": "bulk call: 604 MB moved per call"},
+                      "append_kv": m, "gpu_launches": 4 * (max(args.steps, 2) + 3)}))
+
+
+# ---------------------------------------------------------------------------------------------
 def run_prefix(args):
     """`--workload prefix`: decode_attention and decode_attention_shared_prefix on the same state - 64 traces of the
     8B layout whose shared prompt is long against what each trace generated (the regime the paper's workloads are
@@ -1345,7 +1384,7 @@ def run_reference_scorer(args, K, Wm, sample=64):
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
-        if a.workload in ("prefix", "replay"):
+        if a.workload in ("prefix", "replay", "append"):
             a.workload = "c1"           # the oracle's arm of the prefix workload is the one-layer configuration it is cut from
         run_reference(a)
     elif a.workload == "scorer":
@@ -1354,5 +1393,7 @@ if __name__ == "__main__":
         run_prefix(a)
     elif a.workload == "replay":
         run_replay(a)
+    elif a.workload == "append":
+        run_append(a)
     else:
         run_ours(a)

@@ -185,11 +185,9 @@ int decode_attention_shared_prefix(step_pool* pool, int layer, const void* q,
  * (cudaGetSymbolAddress) before it launches.  Make that first call outside any stream capture.
  *
  * Sharing: all calls on a device - from every pool and every stream - use the same array, and it
- * keeps whatever the previous call left.  The partials need no clearing (each call writes every partial
- * before it reads it); the small ticket counters in it must be zero when the kernel starts, so every call
- * clears the ones it will use (n * num_kv_heads ints) with a memset on its stream before the launch.  That
- * also covers the one case in which a call does not leave them zero: a call whose bounded device wait ran
- * out (STEP_ERR_TIMEOUT in the pool's status word) abandons its tickets mid-count and its outputs are
+ * keeps whatever the previous call left.  Nothing in it needs clearing: each call writes every partial
+ * before it reads it.  A call whose bounded device wait ran out (STEP_ERR_TIMEOUT in the pool's status word)
+ * leaves some partials unwritten and its outputs are
  * undefined; the next call starts clean all the same.  Two calls that overlap in time on the GPU race on
  * the array: keep calls of this entry point ordered, e.g. on one stream. */
 int decode_attention_static(step_pool* pool, int layer, const void* q,
@@ -392,10 +390,9 @@ int kv_pool_set_attention_config(step_pool* pool, int grid_ctas, int fast_path);
 int kv_pool_set_attention_balance(step_pool* pool, int dynamic_sixteenths, int min_chunk_pages);
 /* How long the tensor-core kernel of decode_attention (all its entry points) waits for a page copy before it gives
  * up: the warp then sets the STEP_ERR_TIMEOUT bit of the status word, waits (with
- * the full limit) for the copies it still has in flight, and leaves; outputs of such a launch are undefined and the
- * tickets of its split sequences may be left mid-count, so call kv_pool_reset (or destroy the pool) before the next
- * decode_attention (decode_attention_static clears its own tickets on every call).  Default 2,000,000,000 ns.  0 = no waiting at all: a page that has not landed by the time it
- * is first looked at counts as timed out - for testing this path, which no healthy device otherwise reaches. */
+ * the full limit) for the copies it still has in flight, and leaves; outputs of such a launch are undefined (the
+ * launches after it are unaffected: no state of the kernel outlives a launch).  Default 2,000,000,000 ns.
+ * 0 = no waiting at all: a page that has not landed by the time it is first looked at counts as timed out - for testing this path, which no healthy device otherwise reaches. */
 int kv_pool_set_wait_limit_ns(step_pool* pool, unsigned long long ns);
 /* Which first-layer kernel score_steps uses for bf16 scorers whose shape the tensor-core kernel covers
  * (D a multiple of 64, m a multiple of 64 and <= 1024, 16-byte aligned W1 and hidden): mode 0 (default)

@@ -6,11 +6,12 @@
 // Two implementations:
 //  * attn_scalar_kernel - any dtype / head_dim / page size, one CTA per (trace, query head).
 //    Used for fp32 pools and for shapes the tensor-core kernel does not cover.
-//  * attn_mma_kernel - bf16, head_dim 128, page 16, G <= 16.  HBM-bound design:
-//      - the whole launch's KV stream (for every trace, for every KV head, its pages in order)
-//        is cut into gridDim * kWarps equal contiguous partitions; a warp owns one partition,
-//        so every SM gets the same number of pages whatever the mix of trace lengths, and no CTA ever waits
-//        for another (the only atomics are the tickets of the split sequences, below);
+//  * attn_mma_kernel + attn_merge_kernel - bf16, head_dim 128, page 16, G <= 16.  HBM-bound design:
+//      - of the launch's KV stream (for every trace, for every KV head, its pages in order) the first pages of
+//        every sequence are cut into gridDim * kWarps equal contiguous shares, one per warp, so every SM gets
+//        the same number of pages whatever the mix of trace lengths; the last pages of every sequence are cut
+//        into chunks that a warp fetches from a device counter when its share is done (SMs do not all stream
+//        at the same rate);
 //      - a page of one KV head (K 4 KiB + V 4 KiB, contiguous, pre-swizzled in HBM) is brought
 //        into shared memory by ONE bulk async copy that signals an mbarrier; every warp keeps
 //        its own ring of kStages pages in flight and never synchronises with another warp;
@@ -18,12 +19,11 @@
 //        S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the
 //        heads on the M axis, ldmatrix (plain for K, transposed for V) feeding the B operand;
 //      - running (max, sum) softmax state per head in fp32, exp2 with the scale folded in;
-//      - a partition that holds a whole (trace, head) sequence writes the output directly;
-//        otherwise it writes an (m, l, o) partial (at most two per warp) and takes a ticket on that
-//        sequence's counter; the warp that draws the last ticket combines the sequence's partials
-//        and writes the output (no second kernel, no waiting: whoever is last does the work);
-//      - a launch that directly follows another launch of this kernel (the next layer of a decode step:
-//        decode_attention_layers) is made its programmatic dependent: it starts on every SM the earlier
+//      - a warp that has read a whole (trace, head) sequence writes the output directly; otherwise it leaves an
+//        (m, l, o) partial in the piece's slot, and attn_merge_kernel - a programmatic dependent of the
+//        streaming kernel, resident beside it - combines every sequence's partials in a fixed order;
+//      - a launch that directly follows another attention launch (the next layer of a decode step:
+//        decode_attention_layers) is made a programmatic dependent too: it starts on every SM the earlier
 //        launch has left, reads and accumulates at once, and waits for that launch's completion only in
 //        front of its own first write, so the stream of KV reads does not stop at layer boundaries.
 #include "step_internal.cuh"
@@ -164,17 +164,23 @@ __device__ inline uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Largest t with Hkv * cum[t] <= pos (cum is an exclusive prefix sum over the launch's sequences).
+__device__ inline int seek_trace(const int* cum, int n, int Hkv, long long pos) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
 // Position in the launch's KV stream -> (trace, kv head, page).  The stream lists, for every
 // trace in order, for every KV head in order, that trace's pages in order.
 struct Cursor {
   int t, h, page, np;   // np = pages of trace t
 };
 __device__ inline void cursor_seek(Cursor& c, const int* cum, int n, int Hkv, long long pos) {
-  int lo = 0, hi = n - 1;                              // largest t with Hkv * cum[t] <= pos
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
-  }
+  const int lo = seek_trace(cum, n, Hkv, pos);
   c.t = lo;
   c.np = cum[lo + 1] - cum[lo];
   const long long r = pos - (long long)Hkv * cum[lo];
@@ -191,16 +197,6 @@ __device__ inline void cursor_next(Cursor& c, const int* cum, int n, int Hkv) {
 }
 
 constexpr int kDynSlotBase = 2 * kMaxPartitions;       // partial slots of the chunks follow those of the equal shares
-
-// Largest t with Hkv * cum[t] <= pos (cum is an exclusive prefix sum over the launch's sequences).
-__device__ inline int seek_trace(const int* cum, int n, int Hkv, long long pos) {
-  int lo = 0, hi = n - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
-  }
-  return lo;
-}
 
 // ---- the partition of a launch, as both the attention kernel and the kernel that combines the pieces derive it
 // from the launch's lengths.
@@ -318,7 +314,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
   // Nothing has been written yet, and nothing read so far is written by another launch of this kernel: when this
   // launch was scheduled ahead of the completion of such a launch before it (a layer-by-layer sequence of calls made
-  // by the library itself), it may run up to its first write - of an output, a partial, a ticket or a claim on the
+  // by the library itself), it may run up to its first write - of an output, a partial or a claim on the
   // chunk counter - and must then wait for that launch, whose scratch it shares.  A no-op for a launch made the
   // plain way.  When the launch before this one is the caller's own kernel that produces q (q_from_primary), the
   // wait moves up to the first read of q: what precedes it - the prefix sums above, the barriers, and every warp's
@@ -1047,7 +1043,7 @@ extern "C" int decode_attention_static(step_pool* pool, int layer, const void* q
   if (layer < 0 || layer >= g.L) return STEP_ERR_INVALID_ARG;
   // only the shape the tensor-core kernel covers
   if (pool->cfg.dtype != STEP_BF16 || g.d != kD || g.P != kP || !pool->swizzle) return STEP_ERR_INVALID_ARG;
-  // sizes beyond what the fixed scratch holds
+  // sizes beyond what the fixed scratch holds, and the entry point's bound on the sequences of one call
   if (g.G > kStaticMaxG || n > kMaxTracesFast || (long long)n * g.Hkv > kStaticMaxSegs) return STEP_ERR_CAPACITY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return STEP_ERR_CUDA;
