@@ -427,7 +427,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
   uint32_t qa[8][4];                 // A fragments of Q for the 8 k-steps over head_dim
   float o_acc[16][4];                // O fragments: 16 n-tiles over head_dim
   float m_run[2], l_run[2];          // rows g_row and g_row + 8
-  int seg_first_page = 0;
+  int seg_first_page = 0, seq_last_page = 0;
   bool seg_open = false, seg_is_first = true;
   int stage = 0;
   uint32_t parity = 0;
@@ -451,9 +451,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
       c_left = cur.cnt;
       seg_open = false; seg_is_first = true;
     }
-    // pages of sequence cc.t in the static stream (a segment of a static share ends there at the latest)
-    const int np_static = s_cum[cc.t + 1] - s_cum[cc.t];
     if (!seg_open) {
+      seq_last_page = s_np[cc.t] - 1;
       // new (trace, head) segment: Q fragments of the G heads of this group, fresh softmax state
       if (a.q_from_primary) before_first_write();
       const uint32_t *q0, *q1;
@@ -496,7 +495,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
 
     // tokens of this page that exist (only the last page of a sequence can be short)
     int valid = kP;
-    if (kMode != kPrefixPass && cc.page == s_np[cc.t] - 1) {    // shared pages are full
+    if (kMode != kPrefixPass && cc.page == seq_last_page) {     // shared pages are full
       int S = a.seq_lens[cc.t];
       const int cap = a.max_pages * kP;
       if (S > cap) S = cap;
@@ -576,10 +575,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
     }
     __syncwarp();
     --in_flight;
-    while (issue_one()) {}                             // refill the stage just consumed
+    issue_one();                                       // refill the stage just consumed
 
     // ---- end of this (trace, head) segment?
-    const bool seq_static_end = !cur.chunk && cc.page + 1 == np_static;
+    // (in a share cc.np counts the sequence's pages in the static stream: a segment ends there at the latest)
+    const bool seq_static_end = !cur.chunk && cc.page + 1 == cc.np;
     const bool seg_end = seq_static_end || c_left == 1;
     if (seg_end) {
       float l0 = l_run[0];
@@ -591,7 +591,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
       }
       // the whole sequence in this one segment: it has no tail, and its static pages lie in this share
-      const bool complete = seq_static_end && seg_first_page == 0 && np_static == s_np[cc.t];
+      const bool complete = seq_static_end && seg_first_page == 0 && cc.page == seq_last_page;
       before_first_write();
       if (complete && kMode == kPrefixPass) {
         // the bundle's whole prefix was read by this warp: (m, l, o) of every (trace, head) row, un-normalised
@@ -664,6 +664,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_mma_kernel(AttnArgs a) {
         // static part that lies inside a single share - there may be many of those in one share - uses the slot of
         // the sequence's spare chunk number.  (A sequence without a tail whose static part lies inside one share
         // was complete and never gets here.)
+        const int np_static = s_cum[cc.t + 1] - s_cum[cc.t];
         const int n_nums = s_cumc[cc.t + 1] - s_cumc[cc.t];
         const int n_ch = n_nums > 0 ? n_nums - 1 : 0;
         const int cbase = Hkv * s_cumc[cc.t] + cc.h * n_nums;
