@@ -134,6 +134,8 @@ def test_random_attention_launches(seed):
         dead = int(g.integers(0, n))
         tw.gpu.release_traces(_dev([dead])); tw.ora.release_trace(dead)
     tw.gpu.set_attention_config(grid_ctas=int(g.integers(1, 149)))
+    # how much of every sequence is handed out at run time, and in how small chunks (0 = equal shares only)
+    tw.gpu.set_attention_balance(int(g.choice([0, 2, 4, 8, 12])), int(g.choice([1, 2, 5, 16])))
     o, v = tw.ora, tw.gpu.views()
     qb, qx = W.normal(cfg.seed, W.TID_Q, (n, hq, 128), "bf16")
     qd = H.to_device(qb, "bf16")
