@@ -493,7 +493,7 @@ def run_ours(args):
         # the same launches counted the way a per-trace kernel would see them (the shared prompt once per trace)
         "kv_gbs_logical": float(np.sum(seq_now - K // 2)) * cfg.bytes_per_token_layer / (attn_avg_ms * 1e-3) / 1e9,
         "attention_share_of_step": float(np.sum(attn_run_ms)) / ms_total,
-        "gpu_launches": K * (2 + 2 * L + 1 + 1), "clocks": clocks,
+        "gpu_launches": K * (1 + 2 * L + 1 + 1), "clocks": clocks,
         "status": {"device_error_mask": err_mask, "live_traces": n_live, "ok": all_ok},
     }
     if e2e:
@@ -701,7 +701,7 @@ def algorithm1_measurement(pool, cfg, T, phys_layers, dev, wts, sets, append_log
     code, bits = pool.last_error()
     return {"iterations": r["iterations"], "ms_per_iteration": ms, "trace_decode_steps_per_s": T / (ms * 1e-3),
             "vs_python_driven_step": None if ms_per_step_python is None else ms_per_step_python / ms,
-            "layers_per_iteration": phys_layers, "launches_per_iteration": 4 + 2 * phys_layers,
+            "layers_per_iteration": phys_layers, "launches_per_iteration": 3 + 2 * phys_layers,
             "live_left": r["live_left"], "n_evicted": r["n_evicted"], "n_finished": r["n_finished"],
             "recorded_iterations": {"iterations": rg["iterations"], "ms_per_iteration": ms_g,
                                     "trace_decode_steps_per_s": T / (ms_g * 1e-3), "vs_direct_launches": ms / ms_g,
@@ -1065,7 +1065,7 @@ def run_append(args):
                       "warmup": 3, "ms_per_step": b["us_per_call_device"] * 1e-3, "higher_is_better": True, "scaling": "weak",
                       "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded, drawn on device)",
                       "config": {"workload": "append_kv on the 64-trace 36-layer layout", "l2_policy": "bulk call: 604 MB moved per call"},
-                      "append_kv": m, "gpu_launches": 4 * (max(args.steps, 2) + 3)}))
+                      "append_kv": m, "gpu_launches": 2 * (max(args.steps, 2) + 3)}))
 
 
 # ---------------------------------------------------------------------------------------------

@@ -172,44 +172,15 @@ fork_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __rest
 }
 
 // ---------------------------------------------------------------- append_kv
-// Phase 1 (one CTA): decide, in list order, which traces get their pages; pop blocks.
+// Two forms.  Pools of up to kFusedMaxTraces traces, and the live-trace form of the Algorithm 1 loop: one launch,
+// append_fused_kernel (further down).  Larger pools: two launches -
+// phase 1 (one CTA): decide, in list order, which traces get their pages; pop blocks.
 // n_dev (may be null): only the first min(n, *n_dev) listed traces take part; the rest are passed over in silence.
-// ids == nullptr (the loop of Algorithm 1, whose row i is trace i): the list is made here first - the live traces
-// among 0 .. n-1 in ascending order go to v.it_ids, and, if tokens is given, those of them whose sampled token is
-// eos go to v.it_fin (the traces that complete in this iteration); the counts to C_IT_NLIVE / C_IT_NFIN.
 __global__ void append_alloc_kernel(DevViews v, Geo g, const int32_t* __restrict__ ids, int n, int n_tokens,
-                                    const int32_t* __restrict__ n_dev, const int32_t* __restrict__ tokens, int eos) {
+                                    const int32_t* __restrict__ n_dev) {
   extern __shared__ int sm[];
   dependents_may_launch();                               // the kernel that writes the rows may set itself up meanwhile
-  int n_listed = -1;
-  if (!ids) {
-    __shared__ int s_cnt[2][8];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int n_live = 0, n_fin = 0;
-    for (int base = 0; base < n; base += blockDim.x) {
-      const int t = base + threadIdx.x;
-      const bool lv = t < n && v.live[t];
-      const bool fin = lv && tokens && tokens[t] == eos;
-      const unsigned bl = __ballot_sync(0xffffffffu, lv), bf = __ballot_sync(0xffffffffu, fin);
-      __syncthreads();                                   // the counts of the pass before have been read
-      if (lane == 0) { s_cnt[0][warp] = __popc(bl); s_cnt[1][warp] = __popc(bf); }
-      __syncthreads();
-      int bl_before = 0, bf_before = 0, bl_all = 0, bf_all = 0;
-      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
-        if (w < warp) { bl_before += s_cnt[0][w]; bf_before += s_cnt[1][w]; }
-        bl_all += s_cnt[0][w]; bf_all += s_cnt[1][w];
-      }
-      const unsigned below = (1u << lane) - 1;
-      if (lv) v.it_ids[n_live + bl_before + __popc(bl & below)] = t;
-      if (fin) v.it_fin[n_fin + bf_before + __popc(bf & below)] = t;
-      n_live += bl_all; n_fin += bf_all;
-    }
-    if (threadIdx.x == 0) { v.counters[C_IT_NLIVE] = n_live; v.counters[C_IT_NFIN] = n_fin; }
-    __syncthreads();                                     // the list is read back below by other threads
-    ids = v.it_ids;
-    n_listed = n_live;
-  }
-  const int n_eff = n_listed >= 0 ? n_listed : (n_dev ? min(n, max(*n_dev, 0)) : n);
+  const int n_eff = n_dev ? min(n, max(*n_dev, 0)) : n;
   int* s_need = sm;            // pages wanted, or -1 if the trace is skipped
   int* s_off = sm + n;         // pops that precede this trace's
   int* s_have = sm + 2 * n;
@@ -304,6 +275,169 @@ append_write_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __re
     const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
     const uint4* src = (which ? vnew : knew) + src_token + r;
     // chunk index of (layer, b, head, which, slot, cdst): pages are [layer][block][head][K|V]
+    const size_t dst0 = (((size_t)b * g.Hkv + head) * 2 + which) * page_chunks + (size_t)slot * cpr + cdst;
+    const size_t layer_stride = (size_t)g.num_blocks * g.Hkv * 2 * page_chunks;
+    for (int l = l0; l < l1; ++l) kv[(size_t)l * layer_stride + dst0] = src[(size_t)l * per_kv];
+  }
+}
+
+// append_kv in ONE launch, for pools of up to kFusedMaxTraces traces (a list's first-place table must fit shared
+// memory; the live-trace form needs none).  grid (listed entries x new tokens, splits of the layer range), as for
+// append_write_kernel; every CTA works out the allocation of the whole call for itself - it is a pure function of the
+// list, the lengths, the live flags and the free count, none of which changes before every CTA has read them:
+//   1. first place of every trace in the list (a repeat is flagged and not served);
+//   2. every entry's length S and page need; sum of the needs in front of this CTA's entry, and of all;
+//      if the free list covers the sum nobody is skipped and entry i pops the blocks
+//      free_list[fc - 1 - before_i - p]; otherwise one thread replays the serial rule (in list order, an entry whose
+//      need exceeds what is left is skipped whole) for exactly the same outcome;
+//   3. a ticket: the CTA that draws the last one knows that every CTA has finished reading, and writes what the
+//      others read - the new lengths, the free count (and, for the live-trace form, the lists of the iteration);
+//   4. the CTA of an entry's first token and first layer range records the entry's new pages (block table, reference
+//      counts); every CTA moves its rows, taking the block of a new page straight from the free list.
+// Nothing waits for anything.
+// ids == nullptr (the loop of Algorithm 1, whose row i is trace i): entry i is trace i and is served if the trace is
+// live; the last CTA also leaves the live traces in ascending order in v.it_ids and, if tokens is given, those of them
+// whose sampled token is eos in v.it_fin (the traces that complete in this iteration), the counts in C_IT_NLIVE /
+// C_IT_NFIN.  n_dev (may be null, lists only): only the first min(n, *n_dev) entries take part.
+constexpr int kFusedMaxTraces = 4096;
+
+__global__ void __launch_bounds__(256)
+append_fused_kernel(DevViews v, Geo g, uint4* __restrict__ kv, const uint4* __restrict__ knew,
+                    const uint4* __restrict__ vnew, const int32_t* __restrict__ ids, int n, int n_tokens,
+                    const int32_t* __restrict__ n_dev, const int32_t* __restrict__ tokens, int eos,
+                    int cpr, int layers_per_cta, int src_by_id) {
+  extern __shared__ int sm[];
+  int* s_S = sm;                 // [n] length before the call; -1: the entry is not served
+  int* s_need = sm + n;          // [n] new pages; -1: not served
+  int* s_first = sm + 2 * n;     // [max_traces] first place in the list that names the trace (lists only)
+  __shared__ int s_red[2][8];
+  __shared__ int s_fc, s_last, s_off, s_granted;
+  const int idx = blockIdx.x / n_tokens, j = blockIdx.x - idx * n_tokens;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool reporter = blockIdx.x == 0 && blockIdx.y == 0;        // raises the status bits (once is enough)
+  const int n_eff = (ids && n_dev) ? min(n, max(*n_dev, 0)) : n;
+  // ---- 1. first places
+  if (ids) {
+    for (int i = threadIdx.x; i < g.max_traces; i += blockDim.x) s_first[i] = 0x7fffffff;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_eff; i += blockDim.x) {
+      const int t = ids[i];
+      if (t >= 0 && t < g.max_traces) atomicMin(&s_first[t], i);
+    }
+    __syncthreads();
+  }
+  // ---- 2. lengths and needs
+  int before = 0, all = 0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    int S = -1, need = -1;
+    if (i < n_eff) {
+      const int t = ids ? ids[i] : i;
+      if (ids) {
+        if (t < 0 || t >= g.max_traces || !v.live[t] || s_first[t] != i) { if (reporter) flag_error(v.counters, STEP_ERR_BAD_TRACE); }
+        else S = v.seq_lens[t];
+      } else if (v.live[t]) {
+        S = v.seq_lens[t];
+      }
+      if (S >= 0) {
+        const int have = (S + g.P - 1) / g.P;
+        const long long want = ((long long)S + n_tokens + g.P - 1) / g.P;
+        if (want > g.max_pages) { if (reporter) flag_error(v.counters, STEP_ERR_CAPACITY); S = -1; }
+        else need = (int)want - have;
+      }
+    }
+    s_S[i] = S; s_need[i] = need;
+    if (need > 0) { all += need; if (i < idx) before += need; }
+  }
+  if (threadIdx.x == 0) s_fc = v.counters[C_FREE_COUNT];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { before += __shfl_xor_sync(0xffffffffu, before, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
+  if (lane == 0) { s_red[0][warp] = before; s_red[1][warp] = all; }
+  __syncthreads();                 // every value this CTA reads from the pool's state has arrived (it sits in shared memory)
+  // ---- 3. the ticket
+  const int total_ctas = gridDim.x * gridDim.y;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = atomicAdd(&v.counters[C_APPEND_TICKET], 1) == total_ctas - 1;
+  }
+  before = 0; all = 0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { before += s_red[0][w]; all += s_red[1][w]; }
+  const int fc = s_fc;
+  if (all > fc) {
+    // the free list cannot serve everybody: the serial rule decides who is skipped
+    if (threadIdx.x == 0) {
+      int remaining = fc, off = 0;
+      for (int i = 0; i < n; ++i) {
+        const int need = s_need[i];
+        if (need < 0) continue;
+        if (need > remaining) { s_need[i] = -1; s_S[i] = -1; if (reporter) flag_error(v.counters, STEP_ERR_NO_BLOCKS); continue; }
+        if (i == idx) off = fc - remaining;
+        remaining -= need;
+      }
+      s_off = off; s_granted = fc - remaining;
+    }
+  } else if (threadIdx.x == 0) {
+    s_off = before; s_granted = all;
+  }
+  __syncthreads();
+  const int S = s_S[idx], need = s_need[idx], off = s_off;
+  const bool served = S >= 0;
+  const int t = ids ? (served ? ids[idx] : 0) : idx;
+  const int have = served ? (S + g.P - 1) / g.P : 0;
+  // ---- 4a. this entry's new pages
+  if (served && j == 0 && blockIdx.y == 0) {
+    int32_t* row = v.block_table + (size_t)t * g.max_pages;
+    for (int p = threadIdx.x; p < need; p += blockDim.x) {
+      const int b = v.free_list[fc - 1 - off - p];
+      row[have + p] = b;
+      v.refcount[b] = 1;
+    }
+  }
+  // ---- 3b. the last CTA to have read writes what was read
+  if (s_last) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+      if (s_S[i] >= 0) v.seq_lens[ids ? ids[i] : i] = s_S[i] + n_tokens;
+    if (threadIdx.x == 0) { v.counters[C_FREE_COUNT] = fc - s_granted; v.counters[C_APPEND_TICKET] = 0; }
+    if (!ids) {
+      // the lists of the Algorithm 1 iteration: traces that were live before this call, and those of them that have
+      // just sampled the end-of-sequence token (ascending ids)
+      __shared__ int s_cnt[2][8];
+      int n_live = 0, n_fin = 0;
+      for (int base = 0; base < n; base += blockDim.x) {
+        const int u = base + threadIdx.x;
+        const bool lv = u < n && v.live[u];
+        const bool fin = lv && tokens && tokens[u] == eos;
+        const unsigned bl = __ballot_sync(0xffffffffu, lv), bf = __ballot_sync(0xffffffffu, fin);
+        __syncthreads();                                 // the counts of the pass before have been read
+        if (lane == 0) { s_cnt[0][warp] = __popc(bl); s_cnt[1][warp] = __popc(bf); }
+        __syncthreads();
+        int bl_before = 0, bf_before = 0, bl_all = 0, bf_all = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+          if (w < warp) { bl_before += s_cnt[0][w]; bf_before += s_cnt[1][w]; }
+          bl_all += s_cnt[0][w]; bf_all += s_cnt[1][w];
+        }
+        const unsigned below = (1u << lane) - 1;
+        if (lv) v.it_ids[n_live + bl_before + __popc(bl & below)] = u;
+        if (fin) v.it_fin[n_fin + bf_before + __popc(bf & below)] = u;
+        n_live += bl_all; n_fin += bf_all;
+      }
+      if (threadIdx.x == 0) { v.counters[C_IT_NLIVE] = n_live; v.counters[C_IT_NFIN] = n_fin; }
+    }
+  }
+  // ---- 4b. the rows
+  if (!served) return;
+  const int pos = S + j, page = pos / g.P, slot = pos % g.P;
+  const int b = page < have ? v.block_table[(size_t)t * g.max_pages + page] : v.free_list[fc - 1 - off - (page - have)];
+  const int l0 = blockIdx.y * layers_per_cta, l1 = min(g.L, l0 + layers_per_cta);
+  const int per_kv = g.Hkv * cpr;                                // chunks of the K (or V) rows of one layer
+  const size_t row = src_by_id ? (size_t)t : (size_t)idx;
+  const size_t src_token = (row * n_tokens + j) * (size_t)g.L * per_kv;
+  const size_t page_chunks = (size_t)g.P * cpr;                  // 16-byte chunks of one K (or V) page
+  for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
+    const int which = i >= per_kv;
+    const int r = which ? i - per_kv : i;
+    const int head = r / cpr, c = r - head * cpr;
+    const int cdst = g.swizzle ? ((c & ~7) | ((c ^ slot) & 7)) : c;
+    const uint4* src = (which ? vnew : knew) + src_token + r;
     const size_t dst0 = (((size_t)b * g.Hkv + head) * 2 + which) * page_chunks + (size_t)slot * cpr + cdst;
     const size_t layer_stride = (size_t)g.num_blocks * g.Hkv * 2 * page_chunks;
     for (int l = l0; l < l1; ++l) kv[(size_t)l * layer_stride + dst0] = src[(size_t)l * per_kv];
@@ -478,8 +612,6 @@ int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int 
   for (int off = 0; off < n; off += kListChunk) {
     const int m = n - off < kListChunk ? n - off : kListChunk;
     if (n_dev && off > 0) return STEP_ERR_INVALID_ARG;              // a device-side count covers one launch only
-    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids ? trace_ids + off : nullptr, m, n_tokens, n_dev,
-                                                                    live_tokens, eos);
     const size_t src_off = src_by_id ? 0 : row_chunks * off;
     // enough CTAs to occupy the device: (trace, token) pairs x splits of the layer range
     const long long pairs = (long long)m * n_tokens;
@@ -489,10 +621,21 @@ int stepk::append_kv_impl(step_pool* pool, const int32_t* trace_ids, int n, int 
     if (splits < 1) splits = 1;
     const int layers_per_cta = (g.L + splits - 1) / splits;
     splits = (g.L + layers_per_cta - 1) / layers_per_cta;
-    // a programmatic dependent of the allocation kernel: scheduled while that one runs, waits for it before its first read
+    if (!trace_ids || g.max_traces <= kFusedMaxTraces) {
+      // one launch does it all
+      const size_t smem = ((size_t)2 * m + (trace_ids ? g.max_traces : 0)) * sizeof(int);
+      append_fused_kernel<<<dim3((unsigned)pairs, (unsigned)splits), 256, smem, s>>>(
+          pool->v, g, (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off, (const uint4*)v_new + src_off,
+          trace_ids ? trace_ids + off : nullptr, m, n_tokens, n_dev, live_tokens, eos, cpr, layers_per_cta, src_by_id);
+      if (launch_ok() != STEP_OK) return STEP_ERR_CUDA;
+      continue;
+    }
+    // larger pools: the allocation in a kernel of its own (its table of first places lives in global memory), the rows
+    // by its programmatic dependent: scheduled while that one runs, waits for it before its first read
+    append_alloc_kernel<<<1, 256, (size_t)m * 3 * sizeof(int), s>>>(pool->v, g, trace_ids + off, m, n_tokens, n_dev);
     if (launch_dependent(append_write_kernel, dim3((unsigned)pairs, (unsigned)splits), dim3(256), 0, s, pool->v, g,
                          (uint4*)pool->cfg.kv_storage, (const uint4*)k_new + src_off, (const uint4*)v_new + src_off,
-                         trace_ids ? trace_ids + off : (const int32_t*)pool->v.it_ids, n_tokens, cpr, layers_per_cta, src_by_id) != cudaSuccess)
+                         trace_ids + off, n_tokens, cpr, layers_per_cta, src_by_id) != cudaSuccess)
       return STEP_ERR_CUDA;
   }
   return launch_ok();

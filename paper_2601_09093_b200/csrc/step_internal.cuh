@@ -38,6 +38,7 @@ enum Counter { C_FREE_COUNT = 0, C_STATUS = 1, C_FORK_OK = 2, C_SCORE_NB = 3, C_
                C_SCORE_TILE = 13,   // rows per work item of the tensor-core scorer kernel (128 or 256)
                C_NEXT_TRACE = 14,   // id the next successful fork starts at
                C_FORK_FIRST = 15,   // first id of the most recent fork (valid when C_FORK_OK is set)
+               C_APPEND_TICKET = 16, // CTAs of the current append launch that have read the pool's state; zero between launches
                C_NUM = 64 };
 
 struct MetaLayout {

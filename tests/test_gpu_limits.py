@@ -77,9 +77,11 @@ def test_prune_list_longer_than_the_shared_memory_staging():
     assert tw.status() == (0, 0)
 
 
-def test_append_list_longer_than_one_launch():
-    """5000 traces in one append_kv call: the list is served in several launches, in list order."""
-    n = 5000
+@pytest.mark.parametrize("n", [5000, 3000])
+def test_append_list_longer_than_one_launch(n):
+    """Thousands of traces in one append_kv call: the list is served in several launches, in list order.  A pool of
+    5000 traces takes the two-launch form of append_kv (allocation kernel, then the rows), one of 3000 the one-launch
+    form; both must follow the serial rule when the free list runs short in the middle of a list, and catch repeats."""
     cfg = W.scaled(W.C0, n_traces=n, prefix_len=16)
     tw = Twin(cfg, n + 64, 3, n, store_payload=False)
     ids, _ = tw.fork(n, 16)
@@ -87,6 +89,18 @@ def test_append_list_longer_than_one_launch():
     assert all(tw.append(order, 1))
     tw.assert_meta_equal()
     assert tw.status() == (0, 0)
+    # 63 blocks are left and every trace wants one more page: the first 63 of the list get theirs
+    served = tw.append(order, 16)
+    assert sum(served) == 63 and all(served[:63])
+    tw.assert_meta_equal()
+    assert tw.status() == (1 << 2, 1 << 2)                        # STEP_ERR_NO_BLOCKS
+    # repeats inside one launch's part of the list are served once
+    short = order[100:140] + order[100:120]
+    z = torch.zeros((len(short), 1, cfg.num_layers, cfg.num_kv_heads, cfg.head_dim), dtype=tw.gpu.torch_dtype, device="cuda")
+    tw.gpu.append_kv(torch.tensor(short, dtype=torch.int32, device="cuda"), 1, z, z)
+    tw.ora.append_kv(order[100:140], 1)
+    tw.assert_meta_equal()
+    assert tw.gpu.last_error()[1] == 1 << 3                        # STEP_ERR_BAD_TRACE
 
 
 def test_scorer_width_2560_on_the_tensor_cores():
