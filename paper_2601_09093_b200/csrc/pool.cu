@@ -515,6 +515,7 @@ int kv_pool_create(const kv_pool_config* cfg, step_pool** out) {
   p->scorer_mode = 0;
   p->scorer_tc_min_rows = 1;
   p->tmap_w1 = nullptr; p->tmap_D = 0; p->tmap_m = 0; p->tc_smem_set = false;
+  p->tmap_h_ptr = nullptr; p->tmap_h_D = 0; p->tmap_h_M = 0;
   p->device = dev;
   p->lay = lay;
   char* m = static_cast<char*>(cfg->meta_storage);

@@ -12,6 +12,8 @@
 //     array, so eight warps gather them with 16-byte cp.async copies straight into the 128-byte-swizzled
 //     K-major arrangement the MMA unit reads (row r of a tile at (r / 8) * 1024 + (r % 8) * 128,
 //     16-byte chunk c stored at chunk c ^ (r % 8)); no compacted copy of the rows is ever made;
+//     when every candidate row is listed (the list is 0, 1, 2, ...) the rows of an item are contiguous in the
+//     caller's array and the TMA thread fetches them as 128-row tiles instead - same arrangement, no gather;
 //   * B = W1[n0 .. n0 + N, k .. k + 64): TMA tiled loads (one 64 x 64 box per 64 units, 128-byte
 //     swizzle) signalling the stage's mbarrier with their byte count;
 //   * the operand ring is 192 KiB; a stage holds exactly what the launch's item shape needs (24 KiB for 128 rows x
@@ -59,6 +61,8 @@ struct TcArgs {
   float* z;
   int32_t* counters;
   int D, m;
+  int Mc;          // candidate rows of the launch
+  int dense_ok;    // the second tensor map describes `hidden` ([Mc, D]): usable when every candidate row is listed
 };
 
 __device__ inline void cp_async16(uint32_t dst, const void* src) {
@@ -125,7 +129,7 @@ __device__ inline uint32_t umma_idesc_bf16(int n) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
+score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_h, TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles want 1024-byte alignment
@@ -197,6 +201,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
     return kHalfRows;
   };
   const int KC = a.D / kBK;
+  // Every candidate row ends a step (scoring collected step-end states offline): the list is 0, 1, 2, ..., the rows
+  // of an item are contiguous in the caller's array, and the TMA thread fetches them as tiles - same arrangement in
+  // shared memory, none of the gather warps' instructions.
+  const bool dense = a.dense_ok && nb == a.Mc;
 
   if (!active) {
     // nothing to do but give the tensor memory back below
@@ -249,7 +257,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
         const int gr = row0 + rb + 32 * i;
         // rows past the end of the list are not fetched: each output row depends on its own operand row only, so
         // whatever the shared memory holds there ends up in accumulator rows that nobody reads out
-        src[i] = gr < nb && 32 * i < rows ? a.hidden + (size_t)a.idx[gr] * a.D + c * 8 : nullptr;
+        src[i] = !dense && gr < nb && 32 * i < rows ? a.hidden + (size_t)a.idx[gr] * a.D + c * 8 : nullptr;
       }
       int kr = first_chunk(item, KC);
       for (int kc = 0; kc < KC; ++kc) {
@@ -279,13 +287,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_w1, TcArgs a) {
       const int boxes = N / kBoxRows;
       for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
         int row0, slice;
-        item_rows(item, row0, slice);
+        const int rows = item_rows(item, row0, slice);
         const int n0 = slice * N;
+        // row halves fetched as tiles (rows past the end of the array arrive as zeros, and count as bytes)
+        const int halves_a = !dense ? 0 : (rows > kHalfRows && row0 + kHalfRows < nb ? 2 : 1);
         int kr = first_chunk(item, KC);
         for (int kc = 0; kc < KC; ++kc) {
           if (*s_abort || !mbar_wait_bounded(bar_empty + 8 * s, ph ^ 1)) { ok = false; break; }
           const uint32_t bar = bar_full + 8 * s;
-          mbar_expect_tx(bar, (uint32_t)(boxes * kBoxBytes));
+          mbar_expect_tx(bar, (uint32_t)(boxes * kBoxBytes + halves_a * kHalfBytes));
+          for (int h = 0; h < halves_a; ++h)
+            tma_load_2d(base + (uint32_t)(s * stage_bytes + h * kHalfBytes), &map_h, kr * kBK, row0 + h * kHalfRows, bar);
           const uint32_t dst = base + (uint32_t)(s * stage_bytes + a_bytes);
           for (int j = 0; j < boxes; ++j) tma_load_2d(dst + j * kBoxBytes, &map_w1, kr * kBK, n0 + j * kBoxRows, bar);
           if (++kr == KC) kr = 0;
@@ -403,6 +415,24 @@ int score_tc_launch(step_pool* pool, const void* hidden, int Mc, const scorer_we
   }
   CUtensorMap map;
   memcpy(&map, pool->tmap_bytes, sizeof(map));
+  // the candidate rows as a [Mc, D] array of 128-row tiles, for launches in which every row ends a step
+  if (pool->tmap_h_ptr != hidden || pool->tmap_h_D != w->D || pool->tmap_h_M != Mc) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return STEP_ERR_CUDA;
+    CUtensorMap fresh;
+    const cuuint64_t dims[2] = {(cuuint64_t)w->D, (cuuint64_t)Mc};
+    const cuuint64_t strides[1] = {(cuuint64_t)w->D * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kHalfRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&fresh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return STEP_ERR_CUDA;
+    memcpy(pool->tmap_h_bytes, &fresh, sizeof(fresh));
+    pool->tmap_h_ptr = hidden; pool->tmap_h_D = w->D; pool->tmap_h_M = Mc;
+  }
+  CUtensorMap map_h;
+  memcpy(&map_h, pool->tmap_h_bytes, sizeof(map_h));
   if (!pool->tc_smem_set) {
     if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
       return STEP_ERR_CUDA;
@@ -413,12 +443,13 @@ int score_tc_launch(step_pool* pool, const void* hidden, int Mc, const scorer_we
   a.b1 = (const __nv_bfloat16*)w->b1; a.w2 = (const __nv_bfloat16*)w->w2;
   a.idx = pool->v.score_idx; a.z = pool->v.score_z; a.counters = pool->v.counters;
   a.D = w->D; a.m = w->m;
+  a.Mc = Mc; a.dense_ok = 1;
   long long max_items = (long long)((Mc + kHalfRows - 1) / kHalfRows) * (w->m / kBoxRows);
   int grid = pool->num_sms;
   if (max_items < grid) grid = (int)max_items;
   if (grid < 1) grid = 1;
   // a dependent launch: the CTAs set themselves up while the compaction kernel is still running
-  if (launch_dependent(score_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, map, a) != cudaSuccess) return STEP_ERR_CUDA;
+  if (launch_dependent(score_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, map, map_h, a) != cudaSuccess) return STEP_ERR_CUDA;
   return launch_ok();
 }
 

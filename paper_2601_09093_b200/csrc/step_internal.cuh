@@ -84,6 +84,9 @@ struct step_pool {
   // the tensor map of the last W1 the tensor-core scorer was given (encoding it costs a few host microseconds)
   alignas(64) unsigned char tmap_bytes[128];
   const void* tmap_w1; int tmap_D, tmap_m;
+  // ... and of the last array of candidate rows it was given
+  alignas(64) unsigned char tmap_h_bytes[128];
+  const void* tmap_h_ptr; int tmap_h_D, tmap_h_M;
   bool tc_smem_set;   // the scorer kernel's dynamic shared memory limit has been raised on this pool's device
   int device;
   stepk::MetaLayout lay;
