@@ -410,6 +410,16 @@ def test_scorer_tensor_core_ragged_tiles_with_row_trace():
     _scorer_case(cfg, M, 1.0 / 16, row_trace=rt, max_score_rows=M, tc_min_rows=100, expect_tc=64)
 
 
+@pytest.mark.parametrize("M", [300, 64 * 40 + 13])
+def test_scorer_tensor_core_every_row_listed_ragged(M):
+    """Every candidate row ends a step, so the tensor-core kernel fetches the rows as tiles of the caller's array
+    instead of gathering them: a second row half that lies partly (or wholly) past the end of the array, several
+    tiles, and a call cut into launches of 1000 rows (each launch sees its own part of the array)."""
+    rt = (np.arange(M) % 64).astype(np.int32)
+    _scorer_case(W.C1, M, 1.0, row_trace=rt, max_score_rows=M, mode=1)
+    _scorer_case(W.C1, M, 1.0, row_trace=rt, max_score_rows=1000, mode=1)
+
+
 def test_scorer_picks_the_cuda_core_kernel_below_the_row_threshold():
     rt = (np.arange(512) % 64).astype(np.int32)
     _scorer_case(W.C1, 512, 1.0 / 8, row_trace=rt, max_score_rows=512, tc_min_rows=128, expect_tc=0)   # ~64 rows
