@@ -9,9 +9,12 @@
 //
 // Parameters, moments and gradients are fp32.  The batch is small (the paper trains with 128 rows), so the two
 // products (B x m x D each) are plain fp32 tiled GEMMs on CUDA cores: forward split over K across CTAs with the
-// partial sums added in a fixed order, backward as a rank-B update with one CTA per 64 x 64 tile of dW1.  Between
+// partial sums added in a fixed order, backward as a rank-B update with one CTA per 64 x 128 tile of dW1, which
+// applies Adam to its tile straight from the accumulators (dW1 is never written out).  Between
 // them a CTA per batch row makes the logit, loss term and dz, and a thread per hidden unit the small gradients.
-// Everything is deterministic (no floating-point atomics).
+// Every output element's sum runs over k (forward: within its K-slice) or over the batch rows (backward) in
+// ascending order with one fused multiply-add per term, whatever the tiling - the order the parameter tolerance
+// against the fp64 oracle was established with.  Everything is deterministic (no floating-point atomics).
 #include "step_internal.cuh"
 
 #include <math.h>
@@ -20,51 +23,73 @@ using namespace stepk;
 
 namespace {
 
-constexpr int kTile = 64, kKStep = 16, kSplitK = 32;   // 32 K-slices: several CTAs per SM hide the load latency
+constexpr int kKStep = 16, kSplitK = 32;               // 32 K-slices: several CTAs per SM hide the load latency
+constexpr int kFwdRows = 128, kFwdUnits = 64;          // forward tile: batch rows x hidden units, 8 x 4 outputs per thread
+constexpr int kBwdUnits = 64, kBwdCols = 128;          // dW1 tile: hidden units x input dims, 4 x 8 outputs per thread
 constexpr int kUnitRows = 16;                          // row slices of train_unit_kernel
 
 template <typename T> __device__ inline float ldf(const T* p);
 template <> __device__ inline float ldf<float>(const float* p) { return *p; }
 template <> __device__ inline float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
+// One Adam step of one parameter (L2 decay folded into the gradient; c1, c2 = 1 - beta^step).
+__device__ __forceinline__ void adam_update(float& w, float& mo, float& va, float g, const scorer_train_hyper& h, float c1, float c2) {
+  g = fmaf(h.weight_decay, w, g);
+  mo = h.beta1 * mo + (1.f - h.beta1) * g;
+  va = h.beta2 * va + (1.f - h.beta2) * g * g;
+  w = w - h.lr * (mo / c1) / (sqrtf(va / c2) + h.eps);
+}
+
 // part[s][b][j] = sum over the s-th slice of k of H[b][k] * W1[j][k].   grid (m tiles, B tiles, kSplitK), 256 threads,
-// a thread owns a 4 x 4 block of the 64 x 64 tile.
+// a thread owns an 8 x 4 block of the 128 x 64 tile: per k, two 16-byte reads of H values and one of W1 values from
+// shared memory feed 32 multiply-adds.
 template <typename T>
 __global__ void __launch_bounds__(256)
 train_fwd_kernel(const T* __restrict__ H, const float* __restrict__ W1, float* __restrict__ part, int B, int D, int m) {
-  __shared__ float sA[kKStep][kTile + 1], sB[kKStep][kTile + 1];
-  const int j0 = blockIdx.x * kTile, b0 = blockIdx.y * kTile;
+  __shared__ __align__(16) float sA[kKStep][kFwdRows + 4], sB[kKStep][kFwdUnits + 4];
+  const int j0 = blockIdx.x * kFwdUnits, b0 = blockIdx.y * kFwdRows;
   const int k_per = (D + kSplitK - 1) / kSplitK;
   const int k_lo = blockIdx.z * k_per, k_hi = min(D, k_lo + k_per);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  float acc[4][4] = {};
+  dependents_may_launch();                               // the row kernel may take its places meanwhile
+  float acc[8][4] = {};
   // the next tile's elements travel in registers while the current tile is multiplied
-  float ra[4], rb[4];
+  float ra[8], rb[4];
   auto fetch = [&](int k0) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = threadIdx.x + q * 256, r = i / kKStep, k = k0 + i % kKStep;
+      ra[q] = (b0 + r < B && k < k_hi) ? ldf(H + (size_t)(b0 + r) * D + k) : 0.f;
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int i = threadIdx.x + q * 256, r = i / kKStep, k = k0 + i % kKStep;
-      ra[q] = (b0 + r < B && k < k_hi) ? ldf(H + (size_t)(b0 + r) * D + k) : 0.f;
       rb[q] = (j0 + r < m && k < k_hi) ? W1[(size_t)(j0 + r) * D + k] : 0.f;
     }
   };
   if (k_lo < k_hi) fetch(k_lo);
   for (int k0 = k_lo; k0 < k_hi; k0 += kKStep) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < 8; ++q) {
       const int i = threadIdx.x + q * 256;
       sA[i % kKStep][i / kKStep] = ra[q];
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = threadIdx.x + q * 256;
       sB[i % kKStep][i / kKStep] = rb[q];
     }
     __syncthreads();
     if (k0 + kKStep < k_hi) fetch(k0 + kKStep);
 #pragma unroll
     for (int kk = 0; kk < kKStep; ++kk) {
-      float av[4], bv[4];
+      const float4 a0 = *reinterpret_cast<const float4*>(&sA[kk][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&sA[kk][ty * 8 + 4]);
+      const float4 bq = *reinterpret_cast<const float4*>(&sB[kk][tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bv[4] = {bq.x, bq.y, bq.z, bq.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { av[i] = sA[kk][ty * 4 + i]; bv[i] = sB[kk][tx * 4 + i]; }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
@@ -72,10 +97,10 @@ train_fwd_kernel(const T* __restrict__ H, const float* __restrict__ W1, float* _
   }
   float* out = part + (size_t)blockIdx.z * B * m;
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int b = b0 + ty * 4 + i, u = j0 + tx * 4 + j;
+      const int b = b0 + ty * 8 + i, u = j0 + tx * 4 + j;
       if (b < B && u < m) out[(size_t)b * m + u] = acc[i][j];
     }
 }
@@ -87,6 +112,8 @@ train_row_kernel(float* __restrict__ part, const float* __restrict__ labels, con
                  float* __restrict__ dz, float* __restrict__ loss_terms) {
   __shared__ float s_red[8];
   const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  dependents_may_launch();
+  wait_for_primary();                                    // the forward product
   float z = 0.f;
   for (int j = threadIdx.x; j < m; j += blockDim.x) {
     const size_t i = (size_t)b * m + j;
@@ -122,6 +149,8 @@ train_unit_kernel(float* __restrict__ part, const float* __restrict__ w2, const 
   __shared__ float s_gw[kUnitRows][32], s_gb[kUnitRows][32];
   const int u = threadIdx.x & 31, r = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + u;
+  dependents_may_launch();
+  wait_for_primary();                                    // the rows' dz
   float gw = 0.f, gb = 0.f;
   if (j < m) {
     const float wj = w2[j];
@@ -148,20 +177,30 @@ train_unit_kernel(float* __restrict__ part, const float* __restrict__ w2, const 
   }
 }
 
-// g_W1[j][k] = sum_b dpre[b][j] * H[b][k].   grid (D tiles, m tiles), 256 threads, 4 x 4 outputs per thread.
+// dW1[j][k] = sum_b dpre[b][j] * H[b][k], and Adam on W1 with it.   grid (D tiles, m tiles), 256 threads, 4 x (4 + 4)
+// outputs of the 64 x 128 tile per thread; the gradient goes from the accumulators straight into the update of W1 and its
+// moments (W1 is not read by this kernel's products, and the forward pass that read it is over).
 template <typename T>
 __global__ void __launch_bounds__(256)
-train_bwd_kernel(const float* __restrict__ dpre, const T* __restrict__ H, float* __restrict__ g_W1, int B, int D, int m) {
-  __shared__ float sA[kKStep][kTile + 1], sB[kKStep][kTile + 1];
-  const int k0 = blockIdx.x * kTile, j0 = blockIdx.y * kTile;
+train_bwd_adam_kernel(const float* __restrict__ dpre, const T* __restrict__ H, float* __restrict__ W1,
+                      float* __restrict__ mom, float* __restrict__ var, int B, int D, int m, scorer_train_hyper h,
+                      float c1, float c2) {
+  __shared__ __align__(16) float sA[kKStep][kBwdUnits + 4], sB[kKStep][kBwdCols + 4];
+  const int k0 = blockIdx.x * kBwdCols, j0 = blockIdx.y * kBwdUnits;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  float acc[4][4] = {};
-  float ra[4], rb[4];
+  float acc[4][8] = {};
+  float ra[4], rb[8];
+  // (a dependent of the small Adam kernel, which has itself waited for the kernel that leaves dpre)
+  wait_for_primary();
   auto fetch = [&](int r0) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const int i = threadIdx.x + q * 256, b = r0 + i / kTile, c = i % kTile;
+      const int i = threadIdx.x + q * 256, b = r0 + i / kBwdUnits, c = i % kBwdUnits;
       ra[q] = (b < B && j0 + c < m) ? dpre[(size_t)b * m + j0 + c] : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = threadIdx.x + q * 256, b = r0 + i / kBwdCols, c = i % kBwdCols;
       rb[q] = (b < B && k0 + c < D) ? ldf(H + (size_t)b * D + k0 + c) : 0.f;
     }
   };
@@ -170,56 +209,86 @@ train_bwd_kernel(const float* __restrict__ dpre, const T* __restrict__ H, float*
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int i = threadIdx.x + q * 256;
-      sA[i / kTile][i % kTile] = ra[q];
-      sB[i / kTile][i % kTile] = rb[q];
+      sA[i / kBwdUnits][i % kBwdUnits] = ra[q];
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = threadIdx.x + q * 256;
+      sB[i / kBwdCols][i % kBwdCols] = rb[q];
     }
     __syncthreads();
     if (r0 + kKStep < B) fetch(r0 + kKStep);
 #pragma unroll
     for (int rr = 0; rr < kKStep; ++rr) {
-      float av[4], bv[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { av[i] = sA[rr][ty * 4 + i]; bv[i] = sB[rr][tx * 4 + i]; }
+      const float4 aq = *reinterpret_cast<const float4*>(&sA[rr][ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&sB[rr][tx * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&sB[rr][kBwdCols / 2 + tx * 4]);
+      const float av[4] = {aq.x, aq.y, aq.z, aq.w};
+      const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
     __syncthreads();
   }
+  // this thread's outputs: rows j0 + 4 ty + i, columns k0 + 4 tx + (0..3) and k0 + 64 + 4 tx + (0..3) - so that the
+  // sixteen threads of a row group touch 256 contiguous bytes of W1 and of each moment at a time
+  const bool vec = D % 4 == 0;
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 4; ++i) {
+    const int u = j0 + ty * 4 + i;
+    if (u >= m) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int u = j0 + ty * 4 + i, k = k0 + tx * 4 + j;
-      if (u < m && k < D) g_W1[(size_t)u * D + k] = acc[i][j];
+    for (int half = 0; half < 2; ++half) {
+      const int k = k0 + half * (kBwdCols / 2) + tx * 4;
+      const size_t idx = (size_t)u * D + k;
+      if (vec && k + 3 < D) {
+        float4 w = *reinterpret_cast<const float4*>(W1 + idx);
+        float4 mo = *reinterpret_cast<const float4*>(mom + idx);
+        float4 va = *reinterpret_cast<const float4*>(var + idx);
+        adam_update(w.x, mo.x, va.x, acc[i][half * 4 + 0], h, c1, c2);
+        adam_update(w.y, mo.y, va.y, acc[i][half * 4 + 1], h, c1, c2);
+        adam_update(w.z, mo.z, va.z, acc[i][half * 4 + 2], h, c1, c2);
+        adam_update(w.w, mo.w, va.w, acc[i][half * 4 + 3], h, c1, c2);
+        *reinterpret_cast<float4*>(W1 + idx) = w;
+        *reinterpret_cast<float4*>(mom + idx) = mo;
+        *reinterpret_cast<float4*>(var + idx) = va;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (k + j >= D) continue;
+          float w = W1[idx + j], mo = mom[idx + j], va = var[idx + j];
+          adam_update(w, mo, va, acc[i][half * 4 + j], h, c1, c2);
+          W1[idx + j] = w; mom[idx + j] = mo; var[idx + j] = va;
+        }
+      }
     }
-}
-
-// Adam over the four parameter tensors laid out one after another: W1 [m*D], b1 [m], w2 [m], b2 [1].
-__global__ void __launch_bounds__(256)
-train_adam_kernel(float* __restrict__ W1, float* __restrict__ b1, float* __restrict__ w2, float* __restrict__ b2,
-                  const float* __restrict__ g_W1, const float* __restrict__ g_b1, const float* __restrict__ g_w2,
-                  const float* __restrict__ g_b2, float* __restrict__ mom, float* __restrict__ var, size_t n_w1, int m,
-                  scorer_train_hyper h, float c1, float c2) {      // c1, c2: 1 - beta^step, worked out on the host
-  const size_t total = n_w1 + 2 * (size_t)m + 1;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    float* p;
-    float g;
-    if (i < n_w1) { p = W1 + i; g = g_W1[i]; }
-    else if (i < n_w1 + m) { p = b1 + (i - n_w1); g = g_b1[i - n_w1]; }
-    else if (i < n_w1 + 2 * (size_t)m) { p = w2 + (i - n_w1 - m); g = g_w2[i - n_w1 - m]; }
-    else { p = b2; g = g_b2[0]; }
-    const float w = *p;
-    g = fmaf(h.weight_decay, w, g);
-    const float mi = h.beta1 * mom[i] + (1.f - h.beta1) * g;
-    const float vi = h.beta2 * var[i] + (1.f - h.beta2) * g * g;
-    mom[i] = mi; var[i] = vi;
-    *p = w - h.lr * (mi / c1) / (sqrtf(vi / c2) + h.eps);
   }
 }
 
-struct TrainLayout { size_t part, dz, loss_terms, g_W1, g_b1, g_w2, g_b2, total; };
+// Adam for b1 [m], w2 [m], b2 [1]; their moments follow those of W1 [m * D] in mom / var.
+__global__ void __launch_bounds__(256)
+train_adam_small_kernel(float* __restrict__ b1, float* __restrict__ w2, float* __restrict__ b2,
+                        const float* __restrict__ g_b1, const float* __restrict__ g_w2, const float* __restrict__ g_b2,
+                        float* __restrict__ mom, float* __restrict__ var, size_t n_w1, int m,
+                        scorer_train_hyper h, float c1, float c2) {      // c1, c2: 1 - beta^step, worked out on the host
+  const int total = 2 * m + 1;
+  dependents_may_launch();
+  wait_for_primary();                                    // the small gradients
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    float* p;
+    float g;
+    if (i < m) { p = b1 + i; g = g_b1[i]; }
+    else if (i < 2 * m) { p = w2 + (i - m); g = g_w2[i - m]; }
+    else { p = b2; g = g_b2[0]; }
+    float w = *p, mo = mom[n_w1 + i], va = var[n_w1 + i];
+    adam_update(w, mo, va, g, h, c1, c2);
+    *p = w; mom[n_w1 + i] = mo; var[n_w1 + i] = va;
+  }
+}
+
+struct TrainLayout { size_t part, dz, loss_terms, g_b1, g_w2, g_b2, total; };
 TrainLayout train_layout(int B, int D, int m) {
   TrainLayout l;
   size_t off = 0;
@@ -227,7 +296,6 @@ TrainLayout train_layout(int B, int D, int m) {
   l.part = take((size_t)kSplitK * B * m);
   l.dz = take(B);
   l.loss_terms = take(B);
-  l.g_W1 = take((size_t)m * D);
   l.g_b1 = take(m);
   l.g_w2 = take(m);
   l.g_b2 = take(1);
@@ -260,29 +328,34 @@ int scorer_train_step(const void* hidden, int hidden_dtype, const float* labels,
   float* part = (float*)(ws + l.part);
   float* dz = (float*)(ws + l.dz);
   float* loss_terms = (float*)(ws + l.loss_terms);
-  float* g_W1 = (float*)(ws + l.g_W1);
   float* g_b1 = (float*)(ws + l.g_b1);
   float* g_w2 = (float*)(ws + l.g_w2);
   float* g_b2 = (float*)(ws + l.g_b2);
-  const dim3 gf((m + kTile - 1) / kTile, (B + kTile - 1) / kTile, kSplitK);
-  const dim3 gb((D + kTile - 1) / kTile, (m + kTile - 1) / kTile);
+  const dim3 gf((m + kFwdUnits - 1) / kFwdUnits, (B + kFwdRows - 1) / kFwdRows, kSplitK);
+  const dim3 gb((D + kBwdCols - 1) / kBwdCols, (m + kBwdUnits - 1) / kBwdUnits);
+  const float c1 = (float)(1.0 - pow((double)h->beta1, (double)h->step));
+  const float c2 = (float)(1.0 - pow((double)h->beta2, (double)h->step));
+  const size_t n_w1 = (size_t)m * D;
   if (hidden_dtype == STEP_BF16)
     train_fwd_kernel<__nv_bfloat16><<<gf, 256, 0, s>>>((const __nv_bfloat16*)hidden, W1, part, B, D, m);
   else
     train_fwd_kernel<float><<<gf, 256, 0, s>>>((const float*)hidden, W1, part, B, D, m);
-  train_row_kernel<<<B, 256, 0, s>>>(part, labels, b1, w2, b2, B, m, h->pos_weight, dz, loss_terms);
-  train_unit_kernel<<<(m + 31) / 32, 32 * kUnitRows, 0, s>>>(part, w2, dz, loss_terms, B, m, g_b1, g_w2, g_b2, loss_out);
+  // the four launches behind the forward product are programmatic dependents of one another: each is scheduled while
+  // the one before it drains and waits for it at its top
+  bool ok = launch_dependent(train_row_kernel, dim3(B), dim3(256), 0, s, part, labels, (const float*)b1, (const float*)w2,
+                             (const float*)b2, B, m, h->pos_weight, dz, loss_terms) == cudaSuccess;
+  ok = ok && launch_dependent(train_unit_kernel, dim3((m + 31) / 32), dim3(32 * kUnitRows), 0, s, part, (const float*)w2,
+                              (const float*)dz, (const float*)loss_terms, B, m, g_b1, g_w2, g_b2, loss_out) == cudaSuccess;
+  // (the small tensors first: the unit kernel's w2 and the row kernel's b1 / b2 have been read by now)
+  ok = ok && launch_dependent(train_adam_small_kernel, dim3((2 * m + 1 + 255) / 256), dim3(256), 0, s, b1, w2, b2,
+                              (const float*)g_b1, (const float*)g_w2, (const float*)g_b2, adam_m, adam_v, n_w1, m, *h, c1, c2) == cudaSuccess;
   if (hidden_dtype == STEP_BF16)
-    train_bwd_kernel<__nv_bfloat16><<<gb, 256, 0, s>>>(part, (const __nv_bfloat16*)hidden, g_W1, B, D, m);
+    ok = ok && launch_dependent(train_bwd_adam_kernel<__nv_bfloat16>, gb, dim3(256), 0, s, (const float*)part,
+                                (const __nv_bfloat16*)hidden, W1, adam_m, adam_v, B, D, m, *h, c1, c2) == cudaSuccess;
   else
-    train_bwd_kernel<float><<<gb, 256, 0, s>>>(part, (const float*)hidden, g_W1, B, D, m);
-  const size_t n_w1 = (size_t)m * D;
-  size_t blocks = (n_w1 + 2 * (size_t)m + 1 + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  const float c1 = (float)(1.0 - pow((double)h->beta1, (double)h->step));
-  const float c2 = (float)(1.0 - pow((double)h->beta2, (double)h->step));
-  train_adam_kernel<<<(unsigned)blocks, 256, 0, s>>>(W1, b1, w2, b2, g_W1, g_b1, g_w2, g_b2, adam_m, adam_v, n_w1, m, *h,
-                                                     c1, c2);
+    ok = ok && launch_dependent(train_bwd_adam_kernel<float>, gb, dim3(256), 0, s, (const float*)part, (const float*)hidden,
+                                W1, adam_m, adam_v, B, D, m, *h, c1, c2) == cudaSuccess;
+  if (!ok) return STEP_ERR_CUDA;
   return launch_ok();
 }
 
