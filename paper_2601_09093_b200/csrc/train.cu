@@ -13,8 +13,10 @@
 // applies Adam to its tile straight from the accumulators (dW1 is never written out).  Between
 // them a CTA per batch row makes the logit, loss term and dz, and a thread per hidden unit the small gradients.
 // Every output element's sum runs over k (forward: within its K-slice) or over the batch rows (backward) in
-// ascending order with one fused multiply-add per term, whatever the tiling - the order the parameter tolerance
-// against the fp64 oracle was established with.  Everything is deterministic (no floating-point atomics).
+// ascending order with one fused multiply-add per term, whatever the tiling: in Adam's first steps a gradient entry
+// near zero decides its parameter's direction by its sign, so the order of summation is part of the result that the
+// parameter tolerance (5e-6 against a double-precision run) was established with.  Everything is deterministic (no
+// floating-point atomics).
 #include "step_internal.cuh"
 
 #include <math.h>
